@@ -1,0 +1,200 @@
+/*
+ * Skip-FFN reference oracle -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, obviously-correct CPU statement of what the Skip-FFN decoder
+ * sublayer computes, forward and backward, in double precision.  It shares no
+ * code, header, table or constant with the CUDA library; only tests, the smoke
+ * check and the benchmark's cpu_baseline leg may call it.
+ *
+ * Definition followed (paper section 4.2, "Training speed-up: skip FFN"):
+ *   retained tokens (Eq. 4):  h = h_attn + FFN(h_attn)
+ *   skipped  tokens (Eq. 5):  h = h_attn
+ * FFN body: the paper's backbones are LLaMA-3-8B / Vicuna, and its cost model
+ * (section 6.2: 3*N*C*M multiply-adds; Table 1: 10.5*L*N*C^2 and 5.64 B FFN
+ * parameters) fixes three C x M matrices, i.e. the bias-free SwiGLU
+ *   FFN(x) = ( silu(x W_gate^T) * (x W_up^T) ) W_down^T ,  silu(z) = z / (1 + exp(-z)).
+ * Backward is the exact derivative of that definition (the paper's claim is a
+ * training speed-up, so the vjp is on the path).
+ *
+ * Layouts (all row-major, contiguous):
+ *   x, dout, out, dx : [N, C]      skip_mask : [N] bytes, nonzero = skipped
+ *   W_gate, W_up     : [I, C]      W_down    : [C, I]
+ * Everything is evaluated one token at a time; no compaction, tiling, blocking
+ * or reordering beyond the definition.  OpenMP only spreads independent
+ * iterations (tokens, or intermediate indices i) over host cores.
+ *
+ * Pins (tests/test_oracle_pins.py): pure-Python per-token brute force on tiny
+ * inputs, scalar closed form, W_gate = 0 / W_down = 0 identities, all-kept ==
+ * dense FFN via a library matmul, all-skipped == input, central finite
+ * differences for every gradient, linearity and homogeneity properties, and the
+ * per-layer skip error of Eq. 8.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ascending list of kept token indices (mask byte == 0); returns their count */
+int64_t skipffn_oracle_compact(const uint8_t *skip_mask, int64_t N, int32_t *idx)
+{
+    int64_t nk = 0;
+    for (int64_t t = 0; t < N; ++t)
+        if (skip_mask[t] == 0)
+            idx[nk++] = (int32_t)t;
+    return nk;
+}
+
+static double sigmoid(double z) { return 1.0 / (1.0 + exp(-z)); }
+
+/* g[i], u[i], h[i] of one token (the three SwiGLU intermediates) */
+static void token_intermediates(const double *xt, const double *Wg, const double *Wu,
+                                int64_t C, int64_t I, double *g, double *u, double *h)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < I; ++i) {
+        double sg = 0.0, su = 0.0;
+        for (int64_t c = 0; c < C; ++c) {
+            sg += xt[c] * Wg[i * C + c];
+            su += xt[c] * Wu[i * C + c];
+        }
+        g[i] = sg;
+        u[i] = su;
+        h[i] = sg * sigmoid(sg) * su;
+    }
+}
+
+/* out[t,:] for every token: Eq. 5 for skipped rows, Eq. 4 for the others.
+ * ffn_only != 0 returns FFN(x) alone on kept rows (and 0 on skipped rows). */
+void skipffn_oracle_forward(const double *x, const uint8_t *skip_mask, const double *Wg,
+                            const double *Wu, const double *Wd, int64_t N, int64_t C,
+                            int64_t I, int ffn_only, double *out)
+{
+    double *g = (double *)malloc(sizeof(double) * (size_t)I * 3);
+    double *u = g + I, *h = u + I;
+    for (int64_t t = 0; t < N; ++t) {
+        const double *xt = x + t * C;
+        double *ot = out + t * C;
+        if (skip_mask[t] != 0) {
+            for (int64_t c = 0; c < C; ++c)
+                ot[c] = ffn_only ? 0.0 : xt[c];
+            continue;
+        }
+        token_intermediates(xt, Wg, Wu, C, I, g, u, h);
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < C; ++c) {
+            double y = 0.0;
+            for (int64_t i = 0; i < I; ++i)
+                y += h[i] * Wd[c * I + i];
+            ot[c] = ffn_only ? y : xt[c] + y;
+        }
+    }
+    free(g);
+}
+
+/* Gradients of L = sum(dout * out) w.r.t. x and the three matrices.
+ * dWg, dWu, dWd may be NULL (then only dx is produced); when given they are
+ * overwritten (zeroed first), never accumulated into. */
+void skipffn_oracle_backward(const double *x, const uint8_t *skip_mask, const double *Wg,
+                             const double *Wu, const double *Wd, const double *dout,
+                             int64_t N, int64_t C, int64_t I, double *dx, double *dWg,
+                             double *dWu, double *dWd)
+{
+    double *g = (double *)malloc(sizeof(double) * (size_t)I * 6);
+    double *u = g + I, *h = u + I, *dh = h + I, *dg = dh + I, *du = dg + I;
+    if (dWg) memset(dWg, 0, sizeof(double) * (size_t)I * (size_t)C);
+    if (dWu) memset(dWu, 0, sizeof(double) * (size_t)I * (size_t)C);
+    if (dWd) memset(dWd, 0, sizeof(double) * (size_t)I * (size_t)C);
+    for (int64_t t = 0; t < N; ++t) {
+        const double *xt = x + t * C, *dot = dout + t * C;
+        double *dxt = dx + t * C;
+        if (skip_mask[t] != 0) { /* derivative of the identity */
+            for (int64_t c = 0; c < C; ++c)
+                dxt[c] = dot[c];
+            continue;
+        }
+        token_intermediates(xt, Wg, Wu, C, I, g, u, h);
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < I; ++i) {
+            double s = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                s += dot[c] * Wd[c * I + i];
+            dh[i] = s;
+            double sg = sigmoid(g[i]);
+            du[i] = s * (g[i] * sg);                                   /* d/du of silu(g)*u */
+            dg[i] = s * u[i] * (sg * (1.0 + g[i] * (1.0 - sg)));       /* silu'(g)          */
+            if (dWd)
+                for (int64_t c = 0; c < C; ++c)
+                    dWd[c * I + i] += dot[c] * h[i];
+            if (dWg)
+                for (int64_t c = 0; c < C; ++c)
+                    dWg[i * C + c] += dg[i] * xt[c];
+            if (dWu)
+                for (int64_t c = 0; c < C; ++c)
+                    dWu[i * C + c] += du[i] * xt[c];
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < C; ++c) {
+            double s = 0.0;
+            for (int64_t i = 0; i < I; ++i)
+                s += dg[i] * Wg[i * C + c] + du[i] * Wu[i * C + c];
+            dxt[c] = dot[c] + s;
+        }
+    }
+    free(g);
+}
+
+/* Sampled mode, rows: out[t,:] and dx[t,:] for the listed tokens only (any order,
+ * kept or skipped), written to out_rows / dx_rows [n_tokens, C].  Same per-element
+ * arithmetic as the full functions; dout / dx_rows may be NULL for forward only. */
+void skipffn_oracle_rows(const double *x, const uint8_t *skip_mask, const double *Wg,
+                         const double *Wu, const double *Wd, const double *dout, int64_t C,
+                         int64_t I, const int64_t *tokens, int64_t n_tokens, double *out_rows,
+                         double *dx_rows)
+{
+    for (int64_t k = 0; k < n_tokens; ++k) {
+        int64_t t = tokens[k];
+        uint8_t one = skip_mask[t];
+        skipffn_oracle_forward(x + t * C, &one, Wg, Wu, Wd, 1, C, I, 0, out_rows + k * C);
+        if (dout && dx_rows)
+            skipffn_oracle_backward(x + t * C, &one, Wg, Wu, Wd, dout + t * C, 1, C, I,
+                                    dx_rows + k * C, NULL, NULL, NULL);
+    }
+}
+
+/* Sampled mode, weight gradients: for each listed intermediate index i the exact
+ *   dW_gate[i,:], dW_up[i,:]  (rows, [n_cols, C])  and  dW_down[:,i]  (column, [n_cols, C])
+ * summed over every kept token.  Needs only g, u, dh at index i per token: O(N_kept * C) per i. */
+void skipffn_oracle_dw_columns(const double *x, const uint8_t *skip_mask, const double *Wg,
+                               const double *Wu, const double *Wd, const double *dout,
+                               int64_t N, int64_t C, int64_t I, const int64_t *cols,
+                               int64_t n_cols, double *dWg_rows, double *dWu_rows,
+                               double *dWd_cols)
+{
+#pragma omp parallel for schedule(dynamic)
+    for (int64_t k = 0; k < n_cols; ++k) {
+        int64_t i = cols[k];
+        double *rg = dWg_rows + k * C, *ru = dWu_rows + k * C, *rd = dWd_cols + k * C;
+        for (int64_t c = 0; c < C; ++c)
+            rg[c] = ru[c] = rd[c] = 0.0;
+        for (int64_t t = 0; t < N; ++t) {
+            if (skip_mask[t] != 0)
+                continue;
+            const double *xt = x + t * C, *dot = dout + t * C;
+            double g = 0.0, u = 0.0, dh = 0.0;
+            for (int64_t c = 0; c < C; ++c) {
+                g += xt[c] * Wg[i * C + c];
+                u += xt[c] * Wu[i * C + c];
+                dh += dot[c] * Wd[c * I + i];
+            }
+            double sg = sigmoid(g);
+            double h = g * sg * u;
+            double du = dh * (g * sg);
+            double dg = dh * u * (sg * (1.0 + g * (1.0 - sg)));
+            for (int64_t c = 0; c < C; ++c) {
+                rd[c] += dot[c] * h;
+                rg[c] += dg * xt[c];
+                ru[c] += du * xt[c];
+            }
+        }
+    }
+}

@@ -1,0 +1,280 @@
+"""Pins for the fp64 CPU oracle: it is checked against things other than itself --
+pure-Python brute force, closed forms, identities the paper fixes (Eq. 4 / Eq. 5 / Eq. 8),
+library routines (numpy matmul, torch autograd in fp64) and central finite differences."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+
+RNG = np.random.default_rng(1234)
+
+
+def _rand_case(N, C, I, p_skip=0.5, seed=0):
+    r = np.random.default_rng(seed)
+    x = r.normal(size=(N, C))
+    wg = r.normal(size=(I, C)) * 0.7
+    wu = r.normal(size=(I, C)) * 0.7
+    wd = r.normal(size=(C, I)) * 0.7
+    dout = r.normal(size=(N, C))
+    mask = (r.random(N) < p_skip).astype(np.uint8)
+    return x, mask, wg, wu, wd, dout
+
+
+# ------------------------------------------------------------------ index list
+def test_compact_bruteforce_and_invariants():
+    for seed in range(5):
+        r = np.random.default_rng(seed)
+        for N in (0, 1, 2, 31, 32, 33, 1000):
+            m = (r.random(N) < 0.6).astype(np.uint8) * r.integers(1, 255, size=N).astype(np.uint8)
+            idx = oracle.compact(m)
+            assert idx.dtype == np.int32
+            assert idx.tolist() == [t for t in range(N) if m[t] == 0]
+            assert idx.size == N - np.count_nonzero(m)
+            assert np.all(np.diff(idx) > 0)
+
+
+def test_compact_structured_highres_closed_form():
+    w = wl.config3(C=8, I=8)          # mask layout does not depend on C, I
+    idx = oracle.compact(w.skip_mask)
+    S = 20 + 48 * 48 + 20
+    assert idx.size == 4 * (12 * 24 + 40) == 1312
+    first = idx[idx < S]
+    vis = first[(first >= 20) & (first < 20 + 2304)] - 20
+    assert vis.size == 288
+    assert np.all((vis // 48) % 4 == 0) and np.all((vis % 48) % 2 == 0)
+
+
+# ------------------------------------------------------------------ forward values
+def _py_token(xt, wg, wu, wd):
+    """Pure-Python SwiGLU FFN of one token, written from the definition."""
+    C, I = len(xt), len(wg)
+    h = []
+    for i in range(I):
+        g = sum(xt[c] * wg[i][c] for c in range(C))
+        u = sum(xt[c] * wu[i][c] for c in range(C))
+        h.append(g / (1.0 + math.exp(-g)) * u)
+    return [sum(h[i] * wd[c][i] for i in range(I)) for c in range(C)]
+
+
+@pytest.mark.parametrize("N,C,I", [(5, 4, 6), (7, 3, 2), (4, 8, 12)])
+def test_forward_bruteforce_tiny(N, C, I):
+    x, mask, wg, wu, wd, _ = _rand_case(N, C, I, seed=N + C)
+    mask[0], mask[-1] = 0, 1
+    out = oracle.forward(x, mask, wg, wu, wd)
+    for t in range(N):
+        if mask[t]:
+            assert out[t].tolist() == x[t].tolist()
+        else:
+            y = _py_token(x[t].tolist(), wg.tolist(), wu.tolist(), wd.tolist())
+            np.testing.assert_allclose(out[t], x[t] + np.array(y), rtol=1e-13, atol=1e-13)
+
+
+def test_forward_scalar_closed_form():
+    # C = I = 1: out = x + silu(x*wg) * (x*wu) * wd
+    for xv, g, u, d in [(0.5, 2.0, -3.0, 0.25), (-1.5, 0.3, 0.7, -2.0), (2.0, -1.0, 1.0, 1.0)]:
+        out = oracle.forward([[xv]], [0], [[g]], [[u]], [[d]])
+        z = xv * g
+        want = xv + z / (1 + math.exp(-z)) * (xv * u) * d
+        assert abs(out[0, 0] - want) < 1e-15
+    # a hand-computed value: x=1, wg=0 -> silu(0)=0 -> out = x exactly
+    assert oracle.forward([[1.0]], [0], [[0.0]], [[5.0]], [[7.0]])[0, 0] == 1.0
+    # x=1, wg=ln(3): sigmoid(ln 3) = 3/4 -> silu = 0.75*ln3 ; wu=2, wd=4 -> out = 1 + 6*ln3
+    out = oracle.forward([[1.0]], [0], [[math.log(3.0)]], [[2.0]], [[4.0]])
+    assert abs(out[0, 0] - (1 + 6 * math.log(3.0))) < 1e-14
+
+
+def test_zero_gate_or_zero_down_is_identity():
+    x, mask, wg, wu, wd, _ = _rand_case(6, 5, 7, p_skip=0.3)
+    assert np.array_equal(oracle.forward(x, mask, np.zeros_like(wg), wu, wd), x)
+    assert np.array_equal(oracle.forward(x, mask, wg, wu, np.zeros_like(wd)), x)
+
+
+def test_all_skipped_is_input_bitwise_and_zero_dw():
+    x, _, wg, wu, wd, dout = _rand_case(9, 6, 10)
+    x[2, 3] = np.nan
+    x[4, 0] = -0.0
+    x[5, 1] = np.inf
+    mask = np.full(9, 7, dtype=np.uint8)
+    out = oracle.forward(x, mask, wg, wu, wd)
+    assert out.tobytes() == x.tobytes()
+    dx, dwg, dwu, dwd = oracle.backward(x, mask, wg, wu, wd, dout)
+    assert dx.tobytes() == dout.tobytes()
+    assert not dwg.any() and not dwu.any() and not dwd.any()
+
+
+def test_all_kept_equals_dense_ffn_library_matmul():
+    from scipy.special import expit
+    x, _, wg, wu, wd, _ = _rand_case(33, 24, 40, seed=3)
+    mask = np.zeros(33, dtype=np.uint8)
+    g = x @ wg.T
+    dense = x + (g * expit(g) * (x @ wu.T)) @ wd.T
+    np.testing.assert_allclose(oracle.forward(x, mask, wg, wu, wd), dense, rtol=1e-12, atol=1e-12)
+
+
+def test_masked_dense_restatement_and_skip_error_eq8():
+    """out = x + keep * FFN_dense(x); on a skipped row the dense output differs from the skip
+    output by FFN(x) of that row, whose 2-norm is the per-layer skip error of Eq. 8."""
+    from scipy.special import expit
+    x, mask, wg, wu, wd, _ = _rand_case(21, 16, 28, seed=5)
+    g = x @ wg.T
+    ffn = (g * expit(g) * (x @ wu.T)) @ wd.T
+    keep = (mask == 0)[:, None]
+    out_skip = oracle.forward(x, mask, wg, wu, wd)
+    np.testing.assert_allclose(out_skip, x + keep * ffn, rtol=1e-12, atol=1e-12)
+    out_dense = oracle.forward(x, np.zeros_like(mask), wg, wu, wd)
+    sk = mask != 0
+    np.testing.assert_allclose((out_dense - out_skip)[sk], ffn[sk], rtol=1e-11, atol=1e-12)
+    eps = np.linalg.norm((out_dense - out_skip)[sk], axis=1)
+    np.testing.assert_allclose(eps, np.linalg.norm(ffn[sk], axis=1), rtol=1e-11)
+    # ffn_only mode
+    np.testing.assert_allclose(oracle.forward(x, mask, wg, wu, wd, ffn_only=True), keep * ffn,
+                               rtol=1e-12, atol=1e-12)
+
+
+def test_token_permutation_equivariance_and_homogeneity():
+    x, mask, wg, wu, wd, _ = _rand_case(13, 8, 12, seed=8)
+    perm = np.random.default_rng(0).permutation(13)
+    a = oracle.forward(x, mask, wg, wu, wd)
+    b = oracle.forward(x[perm], mask[perm], wg, wu, wd)
+    np.testing.assert_allclose(b, a[perm], rtol=0, atol=0)
+    c = oracle.forward(x, mask, wg, wu, -2.5 * wd)
+    np.testing.assert_allclose(c - x, -2.5 * (a - x), rtol=1e-12, atol=1e-13)
+
+
+def test_poisoned_skipped_rows_do_not_leak():
+    x, mask, wg, wu, wd, dout = _rand_case(12, 6, 9, seed=11)
+    xp, dp = x.copy(), dout.copy()
+    xp[mask != 0] = np.nan
+    dp[mask != 0] = np.inf
+    a = oracle.forward(x, mask, wg, wu, wd)
+    b = oracle.forward(xp, mask, wg, wu, wd)
+    kept = mask == 0
+    assert np.array_equal(a[kept], b[kept])
+    ga = oracle.backward(x, mask, wg, wu, wd, dout)
+    gb = oracle.backward(xp, mask, wg, wu, wd, dp)
+    assert np.array_equal(ga[0][kept], gb[0][kept])
+    for u, v in zip(ga[1:], gb[1:]):
+        assert np.array_equal(u, v)
+
+
+# ------------------------------------------------------------------ backward values
+def _loss(x, mask, wg, wu, wd, dout):
+    return float(np.sum(dout * oracle.forward(x, mask, wg, wu, wd)))
+
+
+def test_backward_central_finite_differences():
+    N, C, I = 5, 4, 6
+    x, mask, wg, wu, wd, dout = _rand_case(N, C, I, seed=21)
+    mask[:] = [0, 1, 0, 0, 1]
+    dx, dwg, dwu, dwd = oracle.backward(x, mask, wg, wu, wd, dout)
+    eps = 1e-6
+    args = [x, wg, wu, wd]
+    grads = [dx, dwg, dwu, dwd]
+    for k, (a, g) in enumerate(zip(args, grads)):
+        num = np.zeros_like(a)
+        for j in np.ndindex(a.shape):
+            ap, am = a.copy(), a.copy()
+            ap[j] += eps
+            am[j] -= eps
+            cur_p = list(args); cur_p[k] = ap
+            cur_m = list(args); cur_m[k] = am
+            num[j] = (_loss(cur_p[0], mask, *cur_p[1:], dout) - _loss(cur_m[0], mask, *cur_m[1:], dout)) / (2 * eps)
+        np.testing.assert_allclose(g, num, rtol=2e-7, atol=2e-8)
+
+
+def test_backward_matches_fp64_autograd():
+    import torch
+    x, mask, wg, wu, wd, dout = _rand_case(17, 12, 20, seed=31)
+    tx, twg, twu, twd = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (x, wg, wu, wd))
+    keep = torch.tensor((mask == 0).astype(np.float64))[:, None]
+    out = tx + keep * ((torch.nn.functional.silu(tx @ twg.T) * (tx @ twu.T)) @ twd.T)
+    (out * torch.tensor(dout)).sum().backward()
+    dx, dwg, dwu, dwd = oracle.backward(x, mask, wg, wu, wd, dout)
+    for got, want in [(dx, tx.grad), (dwg, twg.grad), (dwu, twu.grad), (dwd, twd.grad)]:
+        np.testing.assert_allclose(got, want.numpy(), rtol=1e-11, atol=1e-12)
+
+
+def test_silu_derivative_via_scalar_case():
+    # C = I = 1, wu = wd = 1, x = 1: out = 1 + silu(wg) ; d out / d wg = silu'(wg)
+    for z in (-3.0, -0.5, 0.0, 0.7, 4.0):
+        _, dwg, _, _ = oracle.backward([[1.0]], [0], [[z]], [[1.0]], [[1.0]], [[1.0]])
+        s = 1 / (1 + math.exp(-z))
+        assert abs(dwg[0, 0] - (s + z * s * (1 - s))) < 1e-15
+        h = 1e-5
+        silu = lambda t: t / (1 + math.exp(-t))
+        assert abs(dwg[0, 0] - (silu(z + h) - silu(z - h)) / (2 * h)) < 1e-9
+
+
+def test_backward_linearity_in_dout_and_skipped_rows():
+    x, mask, wg, wu, wd, d1 = _rand_case(10, 6, 8, seed=41)
+    d2 = np.random.default_rng(5).normal(size=d1.shape)
+    a = oracle.backward(x, mask, wg, wu, wd, d1)
+    b = oracle.backward(x, mask, wg, wu, wd, d2)
+    c = oracle.backward(x, mask, wg, wu, wd, 2 * d1 - 3 * d2)
+    for u, v, w in zip(a, b, c):
+        np.testing.assert_allclose(w, 2 * u - 3 * v, rtol=1e-11, atol=1e-12)
+    sk = mask != 0
+    assert a[0][sk].tobytes() == d1[sk].tobytes()
+    # weight gradients ignore dout on skipped rows entirely
+    d3 = d1.copy()
+    d3[sk] = 123.0
+    e = oracle.backward(x, mask, wg, wu, wd, d3)
+    for u, v in zip(a[1:], e[1:]):
+        assert np.array_equal(u, v)
+
+
+def test_dw_equals_dense_backward_with_masked_ffn_branch():
+    x, mask, wg, wu, wd, dout = _rand_case(14, 6, 10, seed=51)
+    keep = (mask == 0)
+    # dense backward over only the kept rows == skip backward weight grads
+    a = oracle.backward(x, mask, wg, wu, wd, dout)
+    b = oracle.backward(x[keep], np.zeros(keep.sum(), np.uint8), wg, wu, wd, dout[keep])
+    for u, v in zip(a[1:], b[1:]):
+        np.testing.assert_allclose(u, v, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(a[0][keep], b[0], rtol=0, atol=0)
+
+
+# ------------------------------------------------------------------ sampled mode
+def test_sampled_modes_match_full():
+    w = wl.small_case(3, "bf16", 64, 96, 2, 8, 48, 0.75)
+    out = oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down)
+    dx, dwg, dwu, dwd = oracle.backward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down, w.dout)
+    tok = [0, 5, 17, 33, w.N - 1, 20, 21]
+    o_r, dx_r = oracle.rows(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down, w.dout, tok)
+    assert np.array_equal(o_r, out[tok]) and np.array_equal(dx_r, dx[tok])
+    cols = [0, 1, 50, 95]
+    a, b, c = oracle.dw_columns(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down, w.dout, cols)
+    np.testing.assert_allclose(a, dwg[cols], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(b, dwu[cols], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(c, dwd[:, cols].T, rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------ paper closed forms
+def _golden():
+    path = os.path.join(os.path.dirname(__file__), "golden", "llama3_8b_ffn_shape.txt")
+    vals = {}
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split("=")
+            vals[k.strip()] = float(v)
+    return vals
+
+
+def test_paper_table1_fixes_swiglu_shape():
+    g = _golden()
+    C, I, L = wl.SWEEP_SHAPES["llama3-8b"] + (32,)
+    assert round(L * 3 * C * I / 1e9, 2) == g["ffn_params_billion"]          # three C x I matrices
+    assert 3 * I / C == g["ffn_complexity_coeff"]                              # 3 * (M / C) = 10.5
+    assert round(L * (2 * C * C + 2 * C * 1024) / 1e9, 2) == g["attention_params_billion"]
+    w = wl.config2(C=8, I=8)
+    per_seq = w.N // w.B
+    assert per_seq == g["visual_tokens"] + g["text_tokens"]
+    # the oracle's weight shapes are exactly those three matrices
+    x, mask, wg, wu, wd, _ = _rand_case(2, 4, 14)
+    assert wg.size + wu.size + wd.size == g["ffn_macs_per_token_coeff"] * 4 * 14
+    oracle.forward(x, mask, wg, wu, wd)
