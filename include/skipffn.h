@@ -1,0 +1,128 @@
+/*
+ * skipffn.h -- C ABI of libskipffn: the Skip-FFN decoder sublayer on NVIDIA B200 (sm_100a).
+ *
+ * Operation (paper section 4.2, "Training speed-up: skip FFN"):
+ *     retained / text tokens  (Eq. 4):   out[t] = x[t] + FFN(x[t])
+ *     skipped visual tokens   (Eq. 5):   out[t] = x[t]                    (exact identity)
+ * with the bias-free SwiGLU feed-forward network of the paper's LLaMA-3 / Vicuna backbones
+ * (three C x I matrices; section 6.2 cost model 3*N*C*M and Table 1):
+ *     FFN(x) = ( silu(x W_gate^T) * (x W_up^T) ) W_down^T ,   silu(z) = z * sigmoid(z).
+ * The backward pass is the exact vector-Jacobian product of that definition: skipped rows
+ * pass dout through unchanged, kept rows add the FFN's vjp, and the weight gradients are sums
+ * over kept rows only.
+ *
+ * Conventions common to every entry point
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; tensors are contiguous and
+ *     row-major, base addresses 16-byte aligned.  The library allocates no device memory, never
+ *     synchronises the stream and never aborts: every problem is reported as a status code.
+ *   - x, out, dout, dx : [N, C] with N = B*S tokens;  skip_mask : [N] bytes, nonzero = skipped.
+ *   - W_gate, W_up : [I, C];  W_down : [C, I]   (out_features x in_features).
+ *   - Element type is cfg.dtype (bf16: fp32 accumulation on tensor cores; fp32: plain FMA).
+ *   - C and I must be multiples of 8, else SKIPFFN_EUNSUPPORTED.
+ *   - All work is enqueued on `stream`; the kept-token count stays on the device.
+ *   - Device-side problems (a pipeline wait that exceeded its limit) set a status word in the
+ *     workspace; the kernel then exits normally and skipffn_poll reports it.
+ */
+#ifndef SKIPFFN_H_
+#define SKIPFFN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SKIPFFN_OK = 0,
+    SKIPFFN_EINVAL = 1,       /* null pointer, bad shape, misaligned pointer, forward missing */
+    SKIPFFN_EUNSUPPORTED = 2, /* shape outside what the kernels handle */
+    SKIPFFN_EWORKSPACE = 3,   /* workspace too small for max_tokens */
+    SKIPFFN_ECUDA = 4,        /* a CUDA runtime / driver call failed */
+    SKIPFFN_ETIMEOUT = 5      /* a device-side wait hit its limit (reported by skipffn_poll) */
+} skipffn_status;
+
+typedef enum { SKIPFFN_BF16 = 0, SKIPFFN_FP32 = 1 } skipffn_dtype;
+
+/* Which kernels serve the GEMMs.  DEFAULT: tcgen05 tensor-core kernels for bf16, plain-FMA
+ * kernels for fp32.  SIMT: plain-FMA kernels for either dtype (an on-device second opinion). */
+typedef enum { SKIPFFN_PATH_DEFAULT = 0, SKIPFFN_PATH_SIMT = 1 } skipffn_path;
+
+typedef struct {
+    int32_t C;               /* hidden size */
+    int32_t I;               /* intermediate size */
+    int32_t dtype;           /* skipffn_dtype of x, weights, out, dx */
+    int32_t dense;           /* 1: ignore skip_mask, every token takes the FFN (comparator) */
+    int32_t grad_dtype_fp32; /* 1: dW_* are fp32 regardless of dtype */
+    int32_t accumulate_dw;   /* 1: dW += ..., 0: dW is overwritten */
+    int32_t path;            /* skipffn_path */
+    int32_t reserved;        /* must be 0 */
+} skipffn_config;
+
+/* Host-side handle linking one forward call to its backward call.  It points into the caller's
+ * workspace, where the kept-row index list, the compacted rows of x and the SwiGLU
+ * intermediates G, U, H (and dG, dU during backward) live. */
+typedef struct skipffn_saved skipffn_saved;
+
+/* Bytes of device workspace needed for up to max_tokens tokens (0 if cfg is invalid). */
+size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens);
+
+/* Create a handle over `workspace` (device memory, 1024-byte aligned, workspace_bytes long).
+ * Host-only: nothing is launched.  EWORKSPACE if the buffer is too small. */
+skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg,
+                                    void *workspace, size_t workspace_bytes, int64_t max_tokens);
+void skipffn_saved_destroy(skipffn_saved *saved);
+
+/* Mask compaction alone (the retained / skipped split is the same for every decoder layer, so a
+ * caller may build it once): writes the ascending kept-row index list and its length into the
+ * workspace.  A later skipffn_forward with skip_mask == NULL reuses it. */
+skipffn_status skipffn_plan(skipffn_saved *saved, const uint8_t *skip_mask, int64_t N,
+                            void *stream);
+
+/* Forward, Eq. 4 / Eq. 5.  x, out: [B*S, C] (out may alias x); skip_mask: [B*S] bytes or NULL to
+ * reuse the list of the last skipffn_plan / skipffn_forward on this handle (same B*S required);
+ * cu_seqlens: optional int32 HOST array of n_seq+1 offsets of a packed batch (B == 1), checked
+ * for monotonicity and total only -- the FFN is token-wise.  Kept rows of `out` are the fp32 sum
+ * x + FFN(x) rounded once; skipped rows are byte copies of x.  The handle borrows the three
+ * weight pointers until skipffn_backward returns. */
+skipffn_status skipffn_forward(skipffn_saved *saved, const void *x, const uint8_t *skip_mask,
+                               int64_t B, int64_t S, const int32_t *cu_seqlens,
+                               int32_t n_seq, const void *W_gate, const void *W_up,
+                               const void *W_down, void *out, void *stream);
+
+/* Backward of the forward last run on `saved`.  dout, dx: [B*S, C] (dx may alias dout);
+ * dW_gate, dW_up: [I, C]; dW_down: [C, I] in cfg.dtype (fp32 if grad_dtype_fp32), overwritten or
+ * accumulated per cfg.accumulate_dw; any dW pointer may be NULL to skip that gradient.
+ * Skipped rows of dx are byte copies of dout.  With zero kept tokens dW is zero (or untouched
+ * when accumulating). */
+skipffn_status skipffn_backward(const void *dout, skipffn_saved *saved, void *dx, void *dW_gate,
+                                void *dW_up, void *dW_down, void *stream);
+
+/* Device addresses of the kept-row index list (int32, ascending) and of its length. */
+skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
+                                const int32_t **nk_dev);
+
+/* Device addresses of the compacted intermediates of the last forward / backward, each
+ * [round_up(Nk,128), I] in cfg.dtype (rows >= Nk are zero): which = 0 G, 1 U, 2 H, 3 dG, 4 dU;
+ * 5 = kept rows of x [.., C]; 6 = kept rows of dout [.., C]. */
+skipffn_status skipffn_get_intermediate(const skipffn_saved *saved, int32_t which,
+                                        const void **ptr_dev);
+
+/* Synchronises `stream`, then reads the device status word: returns SKIPFFN_ETIMEOUT (and the
+ * site code in *site_out, may be NULL) if a kernel gave up on a wait, SKIPFFN_ECUDA if the
+ * stream reports an error, else SKIPFFN_OK.  The word is cleared. */
+skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_out);
+
+/* Number of kernels the last forward (which=0) or backward (which=1) call enqueued. */
+int32_t skipffn_last_launches(const skipffn_saved *saved, int32_t which);
+
+/* Algorithmic floating-point operations of one forward+backward call with n_kept kept tokens:
+ * 18 * n_kept * C * I (forward 6: three GEMMs of the section 6.2 cost model; backward 12). */
+double skipffn_flops(const skipffn_config *cfg, int64_t n_kept);
+
+const char *skipffn_strerror(skipffn_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SKIPFFN_H_ */

@@ -1,0 +1,254 @@
+"""ctypes binding of the Skip-FFN C ABI (see ``include/skipffn.h`` for the contract)."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+BF16, FP32 = 0, 1
+PATH_DEFAULT, PATH_SIMT = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libskipffn.so")
+_lib: Optional[ctypes.CDLL] = None
+
+# every symbol the header declares
+EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_destroy",
+           "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
+           "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
+           "skipffn_strerror"]
+
+
+class SkipFFNError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {skipffn_strerror(status)} (status {status})")
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("C", ctypes.c_int32), ("I", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("dense", ctypes.c_int32), ("grad_dtype_fp32", ctypes.c_int32),
+                ("accumulate_dw", ctypes.c_int32), ("path", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libskipffn.so`` (built in-tree by ``paper_2503_21817_b200.build.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                           "`python -m paper_2503_21817_b200.build` (there is no fallback path)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    cfgp = ctypes.POINTER(_Config)
+    lib.skipffn_workspace_bytes.restype = ctypes.c_size_t
+    lib.skipffn_workspace_bytes.argtypes = [cfgp, i64]
+    lib.skipffn_saved_create.restype = i32
+    lib.skipffn_saved_create.argtypes = [ctypes.POINTER(vp), cfgp, vp, ctypes.c_size_t, i64]
+    lib.skipffn_saved_destroy.restype = None
+    lib.skipffn_saved_destroy.argtypes = [vp]
+    lib.skipffn_plan.restype = i32
+    lib.skipffn_plan.argtypes = [vp, vp, i64, vp]
+    lib.skipffn_forward.restype = i32
+    lib.skipffn_forward.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, vp]
+    lib.skipffn_backward.restype = i32
+    lib.skipffn_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.skipffn_get_kept.restype = i32
+    lib.skipffn_get_kept.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.skipffn_get_intermediate.restype = i32
+    lib.skipffn_get_intermediate.argtypes = [vp, i32, ctypes.POINTER(vp)]
+    lib.skipffn_poll.restype = i32
+    lib.skipffn_poll.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.skipffn_last_launches.restype = i32
+    lib.skipffn_last_launches.argtypes = [vp, i32]
+    lib.skipffn_flops.restype = ctypes.c_double
+    lib.skipffn_flops.argtypes = [cfgp, i64]
+    lib.skipffn_strerror.restype = ctypes.c_char_p
+    lib.skipffn_strerror.argtypes = [i32]
+    _lib = lib
+    return lib
+
+
+def _cfg(C, I, dtype=BF16, dense=False, grad_fp32=False, accumulate_dw=False, path=PATH_DEFAULT):
+    return _Config(int(C), int(I), int(dtype), int(bool(dense)), int(bool(grad_fp32)),
+                   int(bool(accumulate_dw)), int(path), 0)
+
+
+def skipffn_workspace_bytes(C, I, max_tokens, dtype=BF16) -> int:
+    c = _cfg(C, I, dtype)
+    return int(load_library().skipffn_workspace_bytes(ctypes.byref(c), int(max_tokens)))
+
+
+def skipffn_flops(C, I, n_kept) -> float:
+    c = _cfg(C, I)
+    return float(load_library().skipffn_flops(ctypes.byref(c), int(n_kept)))
+
+
+def skipffn_strerror(status: int) -> str:
+    return load_library().skipffn_strerror(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+class SkipFFN:
+    """One Skip-FFN sublayer context: owns the workspace tensor and the ``skipffn_saved`` handle.
+
+    ``forward`` / ``backward`` / ``plan`` / ``poll`` mirror ``skipffn_forward`` /
+    ``skipffn_backward`` / ``skipffn_plan`` / ``skipffn_poll``; tensors are CUDA tensors whose
+    ``data_ptr()`` is handed to the library, work is enqueued on the current torch stream.
+    """
+
+    def __init__(self, C: int, I: int, max_tokens: int, dtype: int = BF16, dense: bool = False,
+                 grad_fp32: bool = False, accumulate_dw: bool = False, path: int = PATH_DEFAULT,
+                 device="cuda"):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("Skip-FFN needs a CUDA device (sm_100a); there is no CPU path")
+        self._torch = torch
+        self.lib = load_library()
+        self.C, self.I, self.dtype, self.max_tokens = int(C), int(I), int(dtype), int(max_tokens)
+        self.grad_fp32 = bool(grad_fp32) or dtype == FP32
+        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path)
+        self.device = torch.device(device)
+        nbytes = int(self.lib.skipffn_workspace_bytes(ctypes.byref(self.cfg), self.max_tokens))
+        if nbytes == 0:
+            raise SkipFFNError(1, "skipffn_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 1023) // 1024 * 1024
+        self._saved = ctypes.c_void_p()
+        st = self.lib.skipffn_saved_create(ctypes.byref(self._saved), ctypes.byref(self.cfg),
+                                           ctypes.c_void_p(self._ws_ptr), nbytes, self.max_tokens)
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_saved_create")
+        self._keep = []   # tensors the handle borrows between forward and backward
+
+    def __del__(self):
+        if getattr(self, "_saved", None) and self._saved.value:
+            self.lib.skipffn_saved_destroy(self._saved)
+            self._saved = ctypes.c_void_p()
+
+    # ------------------------------------------------------------------ helpers
+    @property
+    def torch_dtype(self):
+        return self._torch.bfloat16 if self.dtype == BF16 else self._torch.float32
+
+    def _stream(self):
+        return ctypes.c_void_p(self._torch.cuda.current_stream(self.device).cuda_stream)
+
+    def _check(self, t, name, shape=None, dtype=None):
+        if t is None:
+            return
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA tensor")
+        if dtype is not None and t.dtype != dtype:
+            raise ValueError(f"{name} must have dtype {dtype}, got {t.dtype}")
+        if shape is not None and tuple(t.shape) != tuple(shape):
+            raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+
+    # ------------------------------------------------------------------ C-ABI mirrors
+    def plan(self, skip_mask):
+        self._check(skip_mask, "skip_mask", dtype=self._torch.uint8)
+        st = self.lib.skipffn_plan(self._saved, _ptr(skip_mask), skip_mask.numel(), self._stream())
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_plan")
+
+    def forward(self, x, skip_mask, W_gate, W_up, W_down, out=None, cu_seqlens=None):
+        """x: [B, S, C] or [N, C]; skip_mask: uint8 [B, S] / [N] or None (reuse the planned list)."""
+        torch, dt = self._torch, self.torch_dtype
+        if x.dim() == 2:
+            B, S = 1, x.shape[0]
+        else:
+            B, S = x.shape[0], x.shape[1]
+        self._check(x, "x", dtype=dt)
+        if x.shape[-1] != self.C:
+            raise ValueError("x has the wrong hidden size")
+        self._check(W_gate, "W_gate", (self.I, self.C), dt)
+        self._check(W_up, "W_up", (self.I, self.C), dt)
+        self._check(W_down, "W_down", (self.C, self.I), dt)
+        if skip_mask is not None:
+            self._check(skip_mask, "skip_mask", dtype=torch.uint8)
+            if skip_mask.numel() != B * S:
+                raise ValueError("skip_mask must have one byte per token")
+        if out is None:
+            out = torch.empty_like(x)
+        self._check(out, "out", x.shape, dt)
+        cu_arr, n_seq = None, 0
+        if cu_seqlens is not None:
+            vals = [int(v) for v in cu_seqlens]
+            n_seq = len(vals) - 1
+            cu_arr = (ctypes.c_int32 * len(vals))(*vals)
+        st = self.lib.skipffn_forward(self._saved, _ptr(x), _ptr(skip_mask), B, S,
+                                      ctypes.cast(cu_arr, ctypes.c_void_p) if cu_arr is not None else None,
+                                      n_seq, _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(out),
+                                      self._stream())
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_forward")
+        self._keep = [W_gate, W_up, W_down]
+        self._shape = tuple(x.shape)
+        return out
+
+    def backward(self, dout, dx=None, dW_gate=None, dW_up=None, dW_down=None, need_dw=True):
+        torch, dt = self._torch, self.torch_dtype
+        self._check(dout, "dout", self._shape, dt)
+        if dx is None:
+            dx = torch.empty_like(dout)
+        self._check(dx, "dx", self._shape, dt)
+        gdt = torch.float32 if self.grad_fp32 else dt
+        if need_dw:
+            if dW_gate is None:
+                dW_gate = torch.empty(self.I, self.C, dtype=gdt, device=self.device)
+            if dW_up is None:
+                dW_up = torch.empty(self.I, self.C, dtype=gdt, device=self.device)
+            if dW_down is None:
+                dW_down = torch.empty(self.C, self.I, dtype=gdt, device=self.device)
+        self._check(dW_gate, "dW_gate", (self.I, self.C), gdt)
+        self._check(dW_up, "dW_up", (self.I, self.C), gdt)
+        self._check(dW_down, "dW_down", (self.C, self.I), gdt)
+        st = self.lib.skipffn_backward(_ptr(dout), self._saved, _ptr(dx), _ptr(dW_gate),
+                                       _ptr(dW_up), _ptr(dW_down), self._stream())
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_backward")
+        return dx, dW_gate, dW_up, dW_down
+
+    def poll(self):
+        """Synchronise the stream and raise if a kernel reported a device-side problem."""
+        site = ctypes.c_int32(0)
+        st = self.lib.skipffn_poll(self._saved, self._stream(), ctypes.byref(site))
+        if st != 0:
+            raise SkipFFNError(st, f"skipffn_poll (site {site.value})")
+
+    def kept(self):
+        """(idx, nk): the ascending kept-row index list as an int32 CUDA tensor view, and Nk."""
+        torch = self._torch
+        idx_p, nk_p = ctypes.c_void_p(), ctypes.c_void_p()
+        st = self.lib.skipffn_get_kept(self._saved, ctypes.byref(idx_p), ctypes.byref(nk_p))
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_get_kept")
+        torch.cuda.current_stream(self.device).synchronize()
+        nk = int(self._view(nk_p.value, 1, torch.int32)[0].item())
+        return self._view(idx_p.value, nk, torch.int32).clone(), nk
+
+    def intermediate(self, which: int, rows: int):
+        """Copy of a compacted intermediate: 0 G, 1 U, 2 H, 3 dG, 4 dU ([rows, I]); 5 Xk, 6 dOk ([rows, C])."""
+        p = ctypes.c_void_p()
+        st = self.lib.skipffn_get_intermediate(self._saved, which, ctypes.byref(p))
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_get_intermediate")
+        cols = self.I if which < 5 else self.C
+        return self._view(p.value, rows * cols, self.torch_dtype).view(rows, cols).clone()
+
+    def _view(self, ptr, numel, dtype):
+        """Tensor view of `numel` elements of the workspace starting at device address `ptr`."""
+        torch = self._torch
+        off = ptr - self.workspace.data_ptr()
+        nbytes = numel * torch.empty(0, dtype=dtype).element_size()
+        return self.workspace[off:off + nbytes].view(dtype)
+
+    def launches(self):
+        return (int(self.lib.skipffn_last_launches(self._saved, 0)),
+                int(self.lib.skipffn_last_launches(self._saved, 1)))

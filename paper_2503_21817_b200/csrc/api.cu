@@ -1,0 +1,324 @@
+// C-ABI entry points of libskipffn: argument checks, workspace layout, launch sequencing.
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace skipffn;
+
+struct skipffn_saved {
+    skipffn_config cfg;
+    int64_t max_tokens, cap;
+    size_t ws_bytes;
+    int esize;
+    // workspace carve-up (device)
+    int32_t *status, *idx, *pos;
+    void *Xk, *dOk, *G, *U, *H, *dG, *dU;
+    // state
+    int64_t planned_N;     // tokens of the current index list, -1 if none
+    int forwarded;
+    const void *Wg, *Wu, *Wd;
+    int launches[2];
+};
+
+namespace {
+
+struct Layout {
+    size_t status, idx, pos, Xk, dOk, G, U, H, dG, dU, total;
+};
+
+bool valid_cfg(const skipffn_config *c)
+{
+    return c && c->C > 0 && c->I > 0 && (c->dtype == SKIPFFN_BF16 || c->dtype == SKIPFFN_FP32) &&
+           (c->path == SKIPFFN_PATH_DEFAULT || c->path == SKIPFFN_PATH_SIMT) && c->reserved == 0;
+}
+
+Layout make_layout(const skipffn_config *c, int64_t max_tokens)
+{
+    Layout l;
+    const int64_t cap = round_up(max_tokens > 0 ? max_tokens : 1, ROW_PAD);
+    const size_t es = c->dtype == SKIPFFN_BF16 ? 2 : 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
+    l.status = take(ST_WORDS * 4);
+    l.idx = take((size_t)cap * 4);
+    l.pos = take((size_t)cap * 4);
+    l.Xk = take((size_t)cap * c->C * es);
+    l.dOk = take((size_t)cap * c->C * es);
+    l.G = take((size_t)cap * c->I * es);
+    l.U = take((size_t)cap * c->I * es);
+    l.H = take((size_t)cap * c->I * es);
+    l.dG = take((size_t)cap * c->I * es);
+    l.dU = take((size_t)cap * c->I * es);
+    l.total = off;
+    return l;
+}
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+bool use_umma(const skipffn_saved *s)
+{
+    return s->cfg.dtype == SKIPFFN_BF16 && s->cfg.path == SKIPFFN_PATH_DEFAULT;
+}
+
+cudaError_t run_gemm(skipffn_saved *s, int which, int epi, const GemmArgs &g, cudaStream_t st)
+{
+    s->launches[which]++;
+    return use_umma(s) ? launch_umma_gemm(epi, g, st) : launch_simt_gemm(epi, s->cfg.dtype, g, st);
+}
+
+GemmArgs base_args(const skipffn_saved *s)
+{
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.status = s->status;
+    g.idx = s->idx;
+    return g;
+}
+
+skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int which, cudaStream_t st)
+{
+    if (N > 0) {
+        s->launches[which]++;
+        if (launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, st) != cudaSuccess)
+            return SKIPFFN_ECUDA;
+    } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
+        return SKIPFFN_ECUDA;
+    }
+    s->planned_N = N;
+    return SKIPFFN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens)
+{
+    if (!valid_cfg(cfg) || max_tokens < 0) return 0;
+    return make_layout(cfg, max_tokens).total;
+}
+
+skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg, void *workspace,
+                                    size_t workspace_bytes, int64_t max_tokens)
+{
+    if (!saved) return SKIPFFN_EINVAL;
+    *saved = nullptr;
+    if (!valid_cfg(cfg) || !workspace || max_tokens < 0) return SKIPFFN_EINVAL;
+    if ((cfg->C % 8) || (cfg->I % 8)) return SKIPFFN_EUNSUPPORTED;
+    if (max_tokens > (int64_t)1 << 30) return SKIPFFN_EUNSUPPORTED;
+    if ((uintptr_t)workspace & 1023u) return SKIPFFN_EINVAL;
+    Layout l = make_layout(cfg, max_tokens);
+    if (workspace_bytes < l.total) return SKIPFFN_EWORKSPACE;
+    skipffn_saved *s = new (std::nothrow) skipffn_saved;
+    if (!s) return SKIPFFN_EINVAL;
+    memset(s, 0, sizeof(*s));
+    s->cfg = *cfg;
+    s->max_tokens = max_tokens;
+    s->cap = round_up(max_tokens > 0 ? max_tokens : 1, ROW_PAD);
+    s->ws_bytes = workspace_bytes;
+    s->esize = cfg->dtype == SKIPFFN_BF16 ? 2 : 4;
+    char *w = (char *)workspace;
+    s->status = (int32_t *)(w + l.status);
+    s->idx = (int32_t *)(w + l.idx);
+    s->pos = (int32_t *)(w + l.pos);
+    s->Xk = w + l.Xk; s->dOk = w + l.dOk;
+    s->G = w + l.G; s->U = w + l.U; s->H = w + l.H; s->dG = w + l.dG; s->dU = w + l.dU;
+    s->planned_N = -1;
+    *saved = s;
+    return SKIPFFN_OK;
+}
+
+void skipffn_saved_destroy(skipffn_saved *saved) { delete saved; }
+
+skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t N, void *stream)
+{
+    if (!s || N < 0 || N > s->max_tokens) return SKIPFFN_EINVAL;
+    if (!skip_mask && !s->cfg.dense && N > 0) return SKIPFFN_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    // the status word is cleared together with the first plan of a handle
+    if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, ST_WORDS * 4, st) != cudaSuccess)
+        return SKIPFFN_ECUDA;
+    s->launches[0] = 0;
+    s->forwarded = 0;
+    return do_plan(s, skip_mask, N, 0, st);
+}
+
+skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
+                               int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
+                               const void *W_gate, const void *W_up, const void *W_down, void *out,
+                               void *stream)
+{
+    if (!s || B < 0 || S < 0) return SKIPFFN_EINVAL;
+    const int64_t N = B * S;
+    if (N > s->max_tokens) return SKIPFFN_EINVAL;
+    if (!W_gate || !W_up || !W_down || (N > 0 && (!x || !out))) return SKIPFFN_EINVAL;
+    if (!aligned16(x) || !aligned16(out) || !aligned16(W_gate) || !aligned16(W_up) || !aligned16(W_down))
+        return SKIPFFN_EINVAL;
+    if (cu_seqlens) {   // packed batch: offsets must be non-decreasing from 0 to N
+        if (n_seq < 0 || cu_seqlens[0] != 0 || cu_seqlens[n_seq] != N) return SKIPFFN_EINVAL;
+        for (int i = 0; i < n_seq; ++i)
+            if (cu_seqlens[i + 1] < cu_seqlens[i]) return SKIPFFN_EINVAL;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const int C = s->cfg.C, I = s->cfg.I;
+    s->forwarded = 0;
+    if (skip_mask || s->cfg.dense) {
+        if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, ST_WORDS * 4, st) != cudaSuccess)
+            return SKIPFFN_ECUDA;
+        s->launches[0] = 0;
+        skipffn_status r = do_plan(s, skip_mask, N, 0, st);
+        if (r != SKIPFFN_OK) return r;
+    } else {
+        if (s->planned_N != N) return SKIPFFN_EINVAL;   // no list to reuse
+        s->launches[0] = 0;
+    }
+    s->Wg = W_gate; s->Wu = W_up; s->Wd = W_down;
+    if (N == 0) { s->forwarded = 1; return SKIPFFN_OK; }
+
+    // kept rows of x -> Xk (also the residual stash when out aliases x); skipped rows -> out
+    RouteArgs r;
+    r.src = x; r.dst_compact = s->Xk; r.dst_identity = out; r.pos = s->pos; r.status = s->status;
+    r.N = N; r.C = C; r.elem_bytes = s->esize;
+    s->launches[0]++;
+    if (launch_route(r, st) != cudaSuccess) return SKIPFFN_ECUDA;
+
+    // G = Xk Wg^T, U = Xk Wu^T, H = silu(G) * U
+    GemmArgs g = base_args(s);
+    g.A = s->Xk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+    g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
+    g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+    g.out0 = s->G; g.out1 = s->U; g.out2 = s->H; g.ldo = I;
+    if (run_gemm(s, 0, EPI_GATEUP, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+
+    // out[idx[r]] = Xk[r] + H Wd^T
+    g = base_args(s);
+    g.A = s->H; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+    g.B = W_down; g.ldb_n = I; g.ldb_k = 1; g.b_outer = C;
+    g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+    g.in0 = s->Xk; g.out0 = out; g.ldo = C;
+    if (run_gemm(s, 0, EPI_DOWN, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    s->forwarded = 1;
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, void *dW_gate,
+                                void *dW_up, void *dW_down, void *stream)
+{
+    if (!s || !s->forwarded) return SKIPFFN_EINVAL;
+    const int64_t N = s->planned_N;
+    if (N > 0 && (!dout || !dx)) return SKIPFFN_EINVAL;
+    if (!aligned16(dout) || !aligned16(dx) || !aligned16(dW_gate) || !aligned16(dW_up) || !aligned16(dW_down))
+        return SKIPFFN_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int C = s->cfg.C, I = s->cfg.I;
+    s->launches[1] = 0;
+    GemmArgs g;
+
+    if (N > 0) {
+        RouteArgs r;
+        r.src = dout; r.dst_compact = s->dOk; r.dst_identity = dx; r.pos = s->pos; r.status = s->status;
+        r.N = N; r.C = C; r.elem_bytes = s->esize;
+        s->launches[1]++;
+        if (launch_route(r, st) != cudaSuccess) return SKIPFFN_ECUDA;
+
+        // dH = dOk Wd ; dG, dU through the activation
+        g = base_args(s);
+        g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+        g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;
+        g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+        g.in0 = s->G; g.in1 = s->U; g.out0 = s->dG; g.out1 = s->dU; g.ldo = I;
+        if (run_gemm(s, 1, EPI_DH, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
+        return SKIPFFN_ECUDA;
+    }
+
+    // weight gradients: reductions over the kept-token axis (K = Nk, read on the device)
+    const int32_t kmax = (int32_t)N;
+    if (dW_down) {   // dWd[c, i] = sum_r dOk[r, c] H[r, i]
+        g = base_args(s);
+        g.A = s->dOk; g.lda_m = 1; g.lda_k = C; g.a_outer = s->cap;
+        g.B = s->H; g.ldb_n = 1; g.ldb_k = I; g.b_outer = s->cap;
+        g.M = C; g.N = I; g.K = kmax; g.k_from_nk = 1;
+        g.out0 = dW_down; g.ldo = I; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
+        if (run_gemm(s, 1, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    }
+    for (int w = 0; w < 2; ++w) {   // dWg[i, c] = sum_r dG[r, i] Xk[r, c]; same for up with dU
+        void *dst = w == 0 ? dW_gate : dW_up;
+        if (!dst) continue;
+        g = base_args(s);
+        g.A = w == 0 ? s->dG : s->dU; g.lda_m = 1; g.lda_k = I; g.a_outer = s->cap;
+        g.B = s->Xk; g.ldb_n = 1; g.ldb_k = C; g.b_outer = s->cap;
+        g.M = I; g.N = C; g.K = kmax; g.k_from_nk = 1;
+        g.out0 = dst; g.ldo = C; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
+        if (run_gemm(s, 1, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    }
+
+    if (N > 0) {   // dx[idx[r]] = dOk[r] + dG Wg + dU Wu
+        g = base_args(s);
+        g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+        g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
+        g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+        g.in0 = s->dOk; g.out0 = dx; g.ldo = C;
+        if (run_gemm(s, 1, EPI_DX, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    }
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev, const int32_t **nk_dev)
+{
+    if (!s || s->planned_N < 0) return SKIPFFN_EINVAL;
+    if (idx_dev) *idx_dev = s->idx;
+    if (nk_dev) *nk_dev = s->status + ST_NK;
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_get_intermediate(const skipffn_saved *s, int32_t which, const void **ptr_dev)
+{
+    if (!s || !ptr_dev) return SKIPFFN_EINVAL;
+    const void *t[7] = {s->G, s->U, s->H, s->dG, s->dU, s->Xk, s->dOk};
+    if (which < 0 || which > 6) return SKIPFFN_EINVAL;
+    *ptr_dev = t[which];
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_poll(skipffn_saved *s, void *stream, int32_t *site_out)
+{
+    if (!s) return SKIPFFN_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SKIPFFN_ECUDA;
+    int32_t w[3] = {0, 0, 0};
+    if (cudaMemcpy(w, s->status, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (site_out) *site_out = w[ST_SITE];
+    if (w[ST_STATUS] != 0) {
+        if (cudaMemset(s->status + ST_STATUS, 0, 8) != cudaSuccess) return SKIPFFN_ECUDA;
+        return (skipffn_status)w[ST_STATUS];
+    }
+    return SKIPFFN_OK;
+}
+
+int32_t skipffn_last_launches(const skipffn_saved *s, int32_t which)
+{
+    return (s && (which == 0 || which == 1)) ? s->launches[which] : -1;
+}
+
+double skipffn_flops(const skipffn_config *cfg, int64_t n_kept)
+{
+    if (!cfg) return 0.0;
+    return 18.0 * (double)n_kept * (double)cfg->C * (double)cfg->I;
+}
+
+const char *skipffn_strerror(skipffn_status st)
+{
+    switch (st) {
+    case SKIPFFN_OK: return "ok";
+    case SKIPFFN_EINVAL: return "invalid argument";
+    case SKIPFFN_EUNSUPPORTED: return "unsupported shape";
+    case SKIPFFN_EWORKSPACE: return "workspace too small";
+    case SKIPFFN_ECUDA: return "CUDA call failed";
+    case SKIPFFN_ETIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

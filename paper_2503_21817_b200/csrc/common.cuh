@@ -1,0 +1,84 @@
+// Shared declarations of the Skip-FFN CUDA library (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "skipffn.h"
+
+namespace skipffn {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status block at the start of the workspace (int32 words).
+enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_WORDS = 64 };
+
+// Wait sites reported through the status word when a bounded wait gives up.
+enum : int { SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_TMEM_EMPTY = 3,
+             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5 };
+
+constexpr int ROW_PAD = 256;   // compacted buffers are zero-padded to this many rows past Nk
+
+static inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float sigmoidf_(float z) { return 1.0f / (1.0f + expf(-z)); }
+
+// h = silu(g) * u  (Eq. 4's FFN body, SwiGLU)
+__device__ __forceinline__ float swiglu(float g, float u) { return g * sigmoidf_(g) * u; }
+
+// Activation backward: given dh and the saved g, u returns dg, du.
+//   du = dh * silu(g);  dg = dh * u * silu'(g),  silu'(g) = s (1 + g (1 - s)),  s = sigmoid(g)
+__device__ __forceinline__ void swiglu_bwd(float dh, float g, float u, float &dg, float &du)
+{
+    float s = sigmoidf_(g);
+    du = dh * (g * s);
+    dg = dh * u * (s * (1.0f + g * (1.0f - s)));
+}
+
+// ---------------------------------------------------------------- launch descriptors (host)
+struct RouteArgs {          // row routing: compact copy of kept rows + identity copy of skipped rows
+    const void *src;        // [N, C]
+    void *dst_compact;      // [cap, C]
+    void *dst_identity;     // [N, C] or nullptr / == src for "nothing to copy"
+    const int32_t *pos;     // [N] rank of token among kept tokens, or -1
+    const int32_t *status;  // status block (Nk)
+    int64_t N;
+    int32_t C;
+    int32_t elem_bytes;
+};
+
+struct GemmArgs {
+    // C[m, n] = sum_k A(m, k) * B(n, k)  (+ second segment A2/B2 when K2 > 0)
+    const void *A, *B, *A2, *B2;
+    int64_t lda_m, lda_k, ldb_n, ldb_k;
+    int64_t a_outer, b_outer;   // addressable rows of the A / B arrays (tensor-map extents)
+    int32_t M, N, K;            // host upper bounds; *_dev overrides when >= 0
+    int32_t m_from_nk, k_from_nk;   // 1: the extent is the device-resident kept count
+    const int32_t *status;      // status block
+    const int32_t *idx;         // kept-row list for scatter epilogues
+    // epilogue operands
+    void *out0, *out1, *out2;   // meaning depends on the epilogue
+    const void *in0, *in1;
+    int64_t ldo;                // leading dimension of outputs
+    int32_t accumulate;         // DW epilogue: add to the destination
+    int32_t out_fp32;           // DW epilogue: destination is float
+};
+
+enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_DX = 4 };
+
+// compact.cu
+cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
+                           int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s);
+cudaError_t launch_route(const RouteArgs &a, cudaStream_t s);
+// simt.cu
+cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
+// umma.cu (bf16 only)
+cudaError_t launch_umma_gemm(int epi, const GemmArgs &a, cudaStream_t s);
+
+}  // namespace skipffn

@@ -1,0 +1,126 @@
+// Mask compaction (kept-row index list) and row routing (gather of kept rows, identity copy of
+// skipped rows).  Integer / byte work only: results are bit-exact by construction.
+#include "common.cuh"
+
+namespace skipffn {
+
+// One CTA of 1024 threads walks the mask in slabs of 16 x 1024 tokens.  Within a slab, token
+// (j, warp, lane) = base + j*1024 + warp*32 + lane; a warp ballot gives each kept token its rank
+// inside its 32-token segment, and an exclusive scan over the 512 segment counts (segments are in
+// ascending token order) gives the segment's offset.  The list is therefore ascending (stable).
+//   idx[r]  : token index of the r-th kept token, r < Nk; entries Nk .. round_up(Nk, ROW_PAD)-1
+//             repeat a valid kept token (or 0) so that padded gathers stay in bounds
+//   pos[t]  : rank of token t among kept tokens, or -1 if skipped
+//   status[ST_NK] = Nk
+constexpr int CP_THREADS = 1024;
+constexpr int CP_J = 16;
+
+__global__ void __launch_bounds__(CP_THREADS)
+k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
+          int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
+{
+    __shared__ int seg[CP_J * 32];
+    __shared__ int slab_total;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    int carry = 0;
+    for (int64_t base = 0; base < N; base += (int64_t)CP_J * CP_THREADS) {
+        unsigned bal[CP_J];
+#pragma unroll
+        for (int j = 0; j < CP_J; ++j) {
+            int64_t t = base + (int64_t)j * CP_THREADS + tid;
+            bool keep = t < N && (dense || mask[t] == 0);
+            bal[j] = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) seg[j * 32 + warp] = __popc(bal[j]);
+        }
+        __syncthreads();
+        if (warp == 0) {   // exclusive scan of the 512 segment counts, 16 per lane
+            int loc[CP_J], sum = 0;
+#pragma unroll
+            for (int q = 0; q < CP_J; ++q) { loc[q] = seg[lane * CP_J + q]; sum += loc[q]; }
+            int incl = sum;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                int v = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += v;
+            }
+            int run = incl - sum;
+#pragma unroll
+            for (int q = 0; q < CP_J; ++q) { seg[lane * CP_J + q] = run; run += loc[q]; }
+            if (lane == 31) slab_total = incl;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < CP_J; ++j) {
+            int64_t t = base + (int64_t)j * CP_THREADS + tid;
+            if (t < N) {
+                if ((bal[j] >> lane) & 1u) {
+                    int r = carry + seg[j * 32 + warp] + __popc(bal[j] & lt);
+                    idx[r] = (int32_t)t;
+                    pos[t] = r;
+                } else {
+                    pos[t] = -1;
+                }
+            }
+        }
+        carry += slab_total;
+        __syncthreads();
+    }
+    // padding entries: repeat the first kept token (any valid row)
+    __shared__ int first;
+    if (tid == 0) { first = carry > 0 ? idx[0] : 0; status[ST_NK] = carry; }
+    __syncthreads();
+    int64_t end = ((int64_t)carry + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+    if (end > cap) end = cap;
+    for (int64_t r = carry + tid; r < end; r += CP_THREADS) idx[r] = first;
+}
+
+cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
+                           int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s)
+{
+    k_compact<<<1, CP_THREADS, 0, s>>>(mask, N, dense, idx, pos, status, cap);
+    return cudaGetLastError();
+}
+
+// Row routing.  Unit u < N is token u: a kept token's row goes to dst_compact[pos[u]], a skipped
+// token's row goes to dst_identity[u] (byte copy; omitted when dst_identity is null or the
+// source itself).  Units u >= N zero the padding rows Nk .. round_up(Nk, ROW_PAD)-1 of
+// dst_compact, which later serve as exact-zero K-padding of the weight-gradient GEMMs.
+constexpr int RT_THREADS = 128;
+
+__global__ void __launch_bounds__(RT_THREADS)
+k_route(const uint4 *__restrict__ src, uint4 *__restrict__ dst_compact,
+        uint4 *__restrict__ dst_identity, const int32_t *__restrict__ pos,
+        const int32_t *__restrict__ status, int64_t N, int row_vecs, int copy_identity)
+{
+    int64_t u = blockIdx.x;
+    if (u < N) {
+        int p = pos[u];
+        const uint4 *s = src + u * row_vecs;
+        uint4 *d;
+        if (p >= 0) d = dst_compact + (int64_t)p * row_vecs;
+        else if (copy_identity) d = dst_identity + u * row_vecs;
+        else return;
+        for (int v = threadIdx.x; v < row_vecs; v += RT_THREADS) d[v] = s[v];
+    } else {
+        int nk = status[ST_NK];
+        int64_t r = nk + (u - N);
+        int64_t end = ((int64_t)nk + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+        if (r >= end) return;
+        uint4 *d = dst_compact + r * row_vecs;
+        for (int v = threadIdx.x; v < row_vecs; v += RT_THREADS) d[v] = make_uint4(0, 0, 0, 0);
+    }
+}
+
+cudaError_t launch_route(const RouteArgs &a, cudaStream_t s)
+{
+    int row_vecs = (int)((int64_t)a.C * a.elem_bytes / 16);
+    int copy_identity = a.dst_identity != nullptr && a.dst_identity != a.src;
+    int64_t units = a.N + ROW_PAD;
+    k_route<<<(unsigned)units, RT_THREADS, 0, s>>>(
+        (const uint4 *)a.src, (uint4 *)a.dst_compact, (uint4 *)a.dst_identity, a.pos, a.status,
+        a.N, row_vecs, copy_identity);
+    return cudaGetLastError();
+}
+
+}  // namespace skipffn

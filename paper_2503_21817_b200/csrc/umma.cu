@@ -1,0 +1,603 @@
+// Tensor-core GEMM kernels of the Skip-FFN path for sm_100a: TMA-fed shared-memory pipeline,
+// tcgen05.mma with fp32 accumulators in tensor memory, fused Skip-FFN epilogues.
+//
+// One persistent kernel template serves every contraction of the path:
+//   C[m, n] = sum_k A(m, k) * B(n, k),   tile 128 (M) x 256 (N) x 64 (K), bf16 in, fp32 accumulate.
+// Either operand may be K-major (global array [rows = M or N, cols = K]) or MN-major (global array
+// [rows = K, cols = M or N]); the latter is what the backward pass needs for W_down (dH), for
+// W_gate / W_up (dX) and for both operands of the weight-gradient GEMMs, whose reduction axis is the
+// compacted token axis.
+//
+// Warp roles (192 threads, one CTA per SM):
+//   warp 0      TMA producer: fills a 4-stage ring of {A 128x64, B 256x64} tiles (128-byte swizzle)
+//   warp 1      MMA issuer: owns the tensor-memory allocation (512 columns = two 128x256 fp32
+//               accumulators), issues four K=16 tcgen05.mma per stage, releases stages and
+//               publishes finished accumulators through tcgen05.commit
+//   warps 2..5  epilogue: read one accumulator (tcgen05.ld, one row per thread) while the MMA warp
+//               fills the other, apply the fused epilogue, write global memory
+//
+// The kept-token count Nk lives in device memory, so tile counts are derived on the device and no
+// host synchronisation sits between mask compaction and the GEMMs.  Every mbarrier wait is
+// bounded: on expiry the CTA records SKIPFFN_ETIMEOUT plus a site code and leaves normally.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace skipffn {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KiB
+constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64-wide MN-major slab of BK rows: 8 KiB
+constexpr int ACC_COLS = 256;                    // fp32 columns per accumulator
+constexpr int TMEM_COLS = 512;
+constexpr int UMMA_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s
+
+// ------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of time).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                            int32_t *status, int site)
+{
+    unsigned long long t0 = globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 0xff) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                if (atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_ETIMEOUT) == 0)
+                    status[ST_SITE] = site;
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int32_t *status, int site)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, site);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
+                 "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; one thread issues for the CTA
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once every tcgen05 operation issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
+// K-major tile:  rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride byte offset).
+// MN-major tile: 64-wide slabs of BK rows x 128 B; 8-row groups 1024 B apart (stride byte offset),
+//                next 64-wide slab CHUNK_BYTES further (leading byte offset).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3fff);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fff) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 256.
+__host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) |
+           ((uint32_t)b_mn_major << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------ kernel
+struct UmmaParams {
+    int32_t M, N, K;                 // host upper bounds
+    int32_t m_from_nk, k_from_nk;    // extent is the device-resident kept count
+    int32_t segments;                // 2: second K segment reads tmA2 / tmB2 (dX)
+    int32_t *status;
+    const int32_t *idx;
+    void *out0, *out1, *out2;
+    const void *in0, *in1;
+    int64_t ldo;
+    int32_t accumulate, out_fp32;
+};
+
+struct alignas(8) SmemCtl {
+    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ void unpack_bf16(uint32_t w, float &lo, float &hi)
+{
+    __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162 *>(&w);
+    lo = __low2float(v);
+    hi = __high2float(v);
+}
+
+template <int EPI, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+            const UmmaParams p)
+{
+    constexpr bool GATEUP = (EPI == EPI_GATEUP);
+    constexpr int N_TILE = GATEUP ? 128 : BN;   // output columns per tile (gate and up share a tile)
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nk = p.status[ST_NK];
+    const int M = p.m_from_nk ? nk : p.M;
+    const int K = p.k_from_nk ? nk : p.K;
+    const int num_m = (M + BM - 1) / BM, num_n = (p.N + N_TILE - 1) / N_TILE;
+    const int num_tiles = num_m * num_n;
+    const int kb_per_seg = (K + BK - 1) / BK;
+    const int num_kb = kb_per_seg * p.segments;
+    const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[s]), 4);
+        }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    volatile int *abort_flag = &ctl->abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && !zero_acc) {
+            prefetch_tmap(&tmA);
+            prefetch_tmap(&tmB);
+            if (GATEUP || p.segments == 2) prefetch_tmap(&tmB2);
+            if (p.segments == 2) prefetch_tmap(&tmA2);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * N_TILE;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status,
+                                   SITE_PRODUCER_EMPTY);
+                    if (!ok) break;
+                    const int seg = kb >= kb_per_seg ? 1 : 0;
+                    const int k0 = (kb - seg * kb_per_seg) * BK;
+                    const CUtensorMap *mA = seg ? &tmA2 : &tmA;
+                    const CUtensorMap *mB = seg ? &tmB2 : &tmB;
+                    const uint32_t bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(bar, STAGE_BYTES);
+                    if (A_MN) {
+#pragma unroll
+                        for (int j = 0; j < BM / 64; ++j)
+                            tma_load_2d(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0, bar);
+                    } else {
+                        tma_load_2d(sa, mA, k0, m0, bar);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j)
+                            tma_load_2d(sb + j * CHUNK_BYTES, mB, n0 + 64 * j, k0, bar);
+                    } else if (GATEUP) {
+                        tma_load_2d(sb, &tmB, k0, n0, bar);                 // 128 gate rows
+                        tma_load_2d(sb + B_BYTES / 2, &tmB2, k0, n0, bar);  // 128 up rows
+                    } else {
+                        tma_load_2d(sb, mB, k0, n0, bar);
+                    }
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && !zero_acc) {
+            constexpr uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0);
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                ok = mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1, abort_flag, p.status,
+                               SITE_MMA_TMEM_EMPTY);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, p.status,
+                                   SITE_MMA_FULL);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        const uint64_t da = A_MN ? make_desc(sa + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
+                                                 : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
+                        const uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
+                                                 : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
+                        umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
+                    }
+                    umma_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(smem_u32(&ctl->tmem_full[acc]));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3;                 // tensor-memory lanes 32*quarter .. +31
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * N_TILE;
+            const int m = m0 + row_in_tile;
+            if (!zero_acc) {
+                ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
+                               SITE_EPI_TMEM_FULL);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
+            const bool row_valid = m < M;
+            int64_t tok = 0;
+            if ((EPI == EPI_DOWN || EPI == EPI_DX) && row_valid) tok = p.idx[m];
+
+#pragma unroll 1
+            for (int c = 0; c < N_TILE / 32; ++c) {
+                const int n = n0 + c * 32;
+                uint32_t r[32], r2[32];
+                if (!zero_acc) {
+                    tmem_ld32(t_row + c * 32, r);
+                    if (GATEUP) tmem_ld32(t_row + 128 + c * 32, r2);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) { r[q] = 0u; r2[q] = 0u; }
+                }
+                if (n >= p.N) continue;
+                const int64_t o = (int64_t)m * p.ldo + n;
+                if (EPI == EPI_GATEUP) {
+                    // compacted G, U, H; rows past Nk inside the tile are written as zeros
+                    bf16 *G = (bf16 *)p.out0 + o, *U = (bf16 *)p.out1 + o, *H = (bf16 *)p.out2 + o;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        if (n + v * 8 >= p.N) break;
+                        uint32_t wg[4], wu[4], wh[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            float g0 = __uint_as_float(r[v * 8 + 2 * q]), g1 = __uint_as_float(r[v * 8 + 2 * q + 1]);
+                            float u0 = __uint_as_float(r2[v * 8 + 2 * q]), u1 = __uint_as_float(r2[v * 8 + 2 * q + 1]);
+                            if (!row_valid) { g0 = g1 = u0 = u1 = 0.0f; }
+                            wg[q] = pack_bf16(g0, g1);
+                            wu[q] = pack_bf16(u0, u1);
+                            wh[q] = pack_bf16(swiglu(g0, u0), swiglu(g1, u1));
+                        }
+                        reinterpret_cast<uint4 *>(G)[v] = make_uint4(wg[0], wg[1], wg[2], wg[3]);
+                        reinterpret_cast<uint4 *>(U)[v] = make_uint4(wu[0], wu[1], wu[2], wu[3]);
+                        reinterpret_cast<uint4 *>(H)[v] = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                    }
+                } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
+                    // residual add in fp32, one rounding, scatter to the token's row
+                    if (row_valid) {
+                        const uint4 *res = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o);
+                        uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)p.out0 + tok * p.ldo + n);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            if (n + v * 8 >= p.N) break;
+                            uint4 rv = res[v];
+                            uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w}, ow[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                float a0, a1;
+                                unpack_bf16(rw[q], a0, a1);
+                                ow[q] = pack_bf16(a0 + __uint_as_float(r[v * 8 + 2 * q]),
+                                                  a1 + __uint_as_float(r[v * 8 + 2 * q + 1]));
+                            }
+                            dst[v] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                        }
+                    }
+                } else if (EPI == EPI_DH) {
+                    const uint4 *Gp = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o);
+                    const uint4 *Up = reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o);
+                    uint4 *dG = reinterpret_cast<uint4 *>((bf16 *)p.out0 + o);
+                    uint4 *dU = reinterpret_cast<uint4 *>((bf16 *)p.out1 + o);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        if (n + v * 8 >= p.N) break;
+                        uint4 gv = make_uint4(0, 0, 0, 0), uv = gv;
+                        if (row_valid) { gv = Gp[v]; uv = Up[v]; }
+                        uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
+                        uint32_t og[4], ou[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            float g0, g1, u0, u1, dg0, dg1, du0, du1;
+                            unpack_bf16(gw[q], g0, g1);
+                            unpack_bf16(uw[q], u0, u1);
+                            swiglu_bwd(__uint_as_float(r[v * 8 + 2 * q]), g0, u0, dg0, du0);
+                            swiglu_bwd(__uint_as_float(r[v * 8 + 2 * q + 1]), g1, u1, dg1, du1);
+                            if (!row_valid) { dg0 = dg1 = du0 = du1 = 0.0f; }
+                            og[q] = pack_bf16(dg0, dg1);
+                            ou[q] = pack_bf16(du0, du1);
+                        }
+                        dG[v] = make_uint4(og[0], og[1], og[2], og[3]);
+                        dU[v] = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+                    }
+                } else {   // EPI_DW: weight-gradient tile, overwrite or accumulate
+                    if (row_valid) {
+                        if (p.out_fp32) {
+                            float4 *dst = reinterpret_cast<float4 *>((float *)p.out0 + o);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                if (n + v * 4 >= p.N) break;
+                                float4 w = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                       __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                                if (p.accumulate) {
+                                    float4 old = dst[v];
+                                    w.x += old.x; w.y += old.y; w.z += old.z; w.w += old.w;
+                                }
+                                dst[v] = w;
+                            }
+                        } else {
+                            uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)p.out0 + o);
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) {
+                                if (n + v * 8 >= p.N) break;
+                                uint32_t ow[4];
+                                uint4 old = make_uint4(0, 0, 0, 0);
+                                if (p.accumulate) old = dst[v];
+                                uint32_t oldw[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    float a0, a1;
+                                    unpack_bf16(oldw[q], a0, a1);
+                                    ow[q] = pack_bf16(a0 + __uint_as_float(r[v * 8 + 2 * q]),
+                                                      a1 + __uint_as_float(r[v * 8 + 2 * q + 1]));
+                                }
+                                dst[v] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                            }
+                        }
+                    }
+                }
+            }
+            if (!zero_acc) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major array [outer, inner] with row pitch `pitch` elements; box = [box_outer, 64].
+// Out-of-range parts of a box read as zero.
+static bool make_map(CUtensorMap *m, const void *base, int64_t inner, int64_t outer, int64_t pitch,
+                     int box_outer)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc || !base) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+    cuuint32_t es[2] = {1u, 1u};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                     box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+static int g_num_sms = 0;
+
+template <int EPI, bool A_MN, bool B_MN>
+static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
+                            const CUtensorMap &b2, const UmmaParams &p, int grid, cudaStream_t s)
+{
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI, A_MN, B_MN>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    k_umma_gemm<EPI, A_MN, B_MN><<<grid, UMMA_THREADS, SMEM_BYTES, s>>>(a, b, a2, b2, p);
+    return cudaGetLastError();
+}
+
+// GemmArgs conventions: an operand with ld_k == 1 is K-major ([outer = M or N rows, inner = K]),
+// otherwise MN-major with ld_mn == 1 ([outer = K rows, inner = M or N]).  a_outer / b_outer give the
+// number of addressable rows of each array.
+cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
+{
+    if (g_num_sms == 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+    }
+    const bool a_mn = g.lda_k != 1, b_mn = g.ldb_k != 1;
+    const bool gateup = epi == EPI_GATEUP;
+    CUtensorMap mA, mB, mA2, mB2;
+    bool ok = true;
+    auto mk = [&](CUtensorMap *m, const void *base, bool mn, int64_t ld_mn, int64_t ld_k,
+                  int64_t mn_extent, int64_t outer_rows, int box_rows_kmajor) {
+        if (mn) return make_map(m, base, mn_extent, outer_rows, ld_k, BK);
+        return make_map(m, base, (int64_t)g.K, outer_rows, ld_mn, box_rows_kmajor);
+    };
+    ok &= mk(&mA, g.A, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM);
+    ok &= mk(&mB, g.B, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, gateup ? 128 : BN);
+    if (g.A2) ok &= mk(&mA2, g.A2, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM); else mA2 = mA;
+    if (g.B2) ok &= mk(&mB2, g.B2, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, gateup ? 128 : BN); else mB2 = mB;
+    if (!ok) return cudaErrorInvalidValue;
+
+    UmmaParams p;
+    p.M = g.M; p.N = g.N; p.K = g.K;
+    p.m_from_nk = g.m_from_nk; p.k_from_nk = g.k_from_nk;
+    p.segments = epi == EPI_DX ? 2 : 1;
+    p.status = const_cast<int32_t *>(g.status);
+    p.idx = g.idx;
+    p.out0 = g.out0; p.out1 = g.out1; p.out2 = g.out2;
+    p.in0 = g.in0; p.in1 = g.in1;
+    p.ldo = g.ldo; p.accumulate = g.accumulate; p.out_fp32 = g.out_fp32;
+
+    const int n_tile = gateup ? 128 : BN;
+    const int64_t max_tiles = ((int64_t)g.M + BM - 1) / BM * (((int64_t)g.N + n_tile - 1) / n_tile);
+    int grid = (int)(max_tiles < g_num_sms ? max_tiles : g_num_sms);
+    if (grid <= 0) return cudaSuccess;
+
+    switch (epi) {
+    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false>(mA, mB, mA2, mB2, p, grid, s);
+    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false>(mA, mB, mA2, mB2, p, grid, s);
+    case EPI_DH:     return launch_k<EPI_DH, false, true>(mA, mB, mA2, mB2, p, grid, s);
+    case EPI_DW:     return launch_k<EPI_DW, true, true>(mA, mB, mA2, mB2, p, grid, s);
+    case EPI_DX:     return launch_k<EPI_DX, false, true>(mA, mB, mA2, mB2, p, grid, s);
+    default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace skipffn

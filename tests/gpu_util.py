@@ -1,0 +1,57 @@
+"""Helpers for the GPU parity tests: move a workload to the device, run the library, fetch results."""
+import numpy as np
+
+import workloads as wl
+
+
+def to_dev(a, dtype):
+    import torch
+    if dtype == "bf16":
+        bits = wl.to_bf16_bits(a).view(np.int16)
+        return torch.from_numpy(bits).cuda().view(torch.bfloat16).reshape(a.shape)
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+
+
+def to_host(t):
+    import torch
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def bits(t):
+    """Raw bytes of a tensor as a numpy array (for bit-exact comparisons)."""
+    import torch
+    return t.detach().contiguous().view(torch.uint8).cpu().numpy()
+
+
+class DeviceWorkload:
+    def __init__(self, w):
+        import torch
+        self.w = w
+        d = w.dtype
+        self.x = to_dev(w.x, d)
+        self.dout = to_dev(w.dout, d)
+        self.W_gate = to_dev(w.W_gate, d)
+        self.W_up = to_dev(w.W_up, d)
+        self.W_down = to_dev(w.W_down, d)
+        self.mask = torch.from_numpy(w.skip_mask).cuda()
+
+
+def run(w, dense=False, path=0, grad_fp32=False, accumulate_dw=False, inplace=False, dev=None,
+        dw_init=None):
+    """Forward + backward through the C ABI; returns a dict of device tensors and the context."""
+    import torch
+    import paper_2503_21817_b200 as sk
+    dev = dev or DeviceWorkload(w)
+    dt = sk.BF16 if w.dtype == "bf16" else sk.FP32
+    ctx = sk.SkipFFN(w.C, w.I, max(w.N, 1), dtype=dt, dense=dense, path=path, grad_fp32=grad_fp32,
+                     accumulate_dw=accumulate_dw)
+    x = dev.x.clone()
+    dout = dev.dout.clone()
+    out = ctx.forward(x, dev.mask, dev.W_gate, dev.W_up, dev.W_down, out=x if inplace else None,
+                      cu_seqlens=w.cu_seqlens)
+    kw = {}
+    if dw_init is not None:
+        kw = dict(dW_gate=dw_init[0], dW_up=dw_init[1], dW_down=dw_init[2])
+    dx, dwg, dwu, dwd = ctx.backward(dout, dx=dout if inplace else None, **kw)
+    ctx.poll()
+    return dict(out=out, dx=dx, dW_gate=dwg, dW_up=dwu, dW_down=dwd, ctx=ctx, dev=dev)
