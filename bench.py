@@ -1,0 +1,337 @@
+#!/usr/bin/env python
+"""Skip-FFN forward+backward benchmark on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg2|cfg3|cfg4|sweep] [--skip-ratio r] [--shape llama3-8b|vicuna-13b]
+
+One step = one pass of the whole hot path (mask compaction, row routing, gate/up GEMM + SiLU*mul,
+down GEMM + residual scatter, and the backward GEMMs dH, dW_down, dW_gate, dW_up, dX) over one
+batch of seeded synthetic input.  Default workload: the LLaMA3-8B-shaped layer, 8 x (576 visual +
+40 text) tokens, 75 % of the visual tokens skipped, bf16 with fp32 accumulation.
+
+Prints ONE JSON line (rank 0).  `value` is kept tokens per second over all ranks with inputs
+resident in HBM; `e2e` is the same metric with the step's inputs copied from pinned host memory
+and its results copied back inside the timed region; `roofline` describes the kernel with the
+largest share of the step; `cpu_baseline` is the fp64 CPU oracle timed on a bounded sample.
+With N > 1 (torchrun) every rank runs an independent replica (no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "skipffn_fwd_bwd_kept_tokens_per_s"
+UNIT = "kept tokens/s"
+KERNEL_NAMES = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
+                "dw_up", "dx"]
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each GEMM kernel at the
+# default workload, from the ncu captures summarised under profiles/; None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def make_workload(args, rank):
+    C, I = wl.SWEEP_SHAPES[args.shape]
+    seed = args.seed + rank
+    if args.workload == "cfg2":
+        return wl.config2(seed=seed, skip_ratio=args.skip_ratio, C=C, I=I)
+    if args.workload == "cfg3":
+        return wl.config3(seed=seed, C=C, I=I)
+    if args.workload == "cfg4":
+        return wl.config4(seed=seed, C=C, I=I)
+    raise ValueError(args.workload)
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.rows = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows]
+        for r in rows:
+            f = [c.strip() for c in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ oracle legs
+def oracle_sample_rate(w, n_tokens):
+    """kept tokens / s of the fp64 CPU oracle (forward + backward, as it stands) on the first
+    `n_tokens` tokens of the workload."""
+    import oracle
+    m = w.skip_mask[:n_tokens]
+    x64, wg, wu, wd, do = (a.astype(np.float64) for a in (w.x[:n_tokens], w.W_gate, w.W_up, w.W_down,
+                                                          w.dout[:n_tokens]))
+    t = time.perf_counter()
+    oracle.forward(x64, m, wg, wu, wd)
+    oracle.backward(x64, m, wg, wu, wd, do)
+    dt = time.perf_counter() - t
+    kept = int((m == 0).sum())
+    return kept / dt, kept, dt, oracle.n_threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, timed step by step on a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args, 0)
+    budget_s = 150.0
+    per_tok = 1.1    # seconds per kept token of this oracle at the 8B shape on ~8 cores (rough)
+    n_tok = int(max(1, min(w.N, budget_s / ((args.steps + args.warmup) * per_tok))))
+    # text tokens lead every sequence and are always kept, so the first tokens are all FFN work
+    rates, kept, cores = [], 0, 0
+    for _ in range(args.warmup):
+        oracle_sample_rate(w, n_tok)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        r, kept, _, cores = oracle_sample_rate(w, n_tok)
+        rates.append(r)
+    total = time.perf_counter() - t0
+    value = kept * args.steps / total
+    sample = f"first {n_tok} tokens of sequence 0 ({kept} kept) per step, full fp64 forward+backward"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(args, w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(args, w):
+    return {"workload": f"{w.name} {args.shape}: C={w.C} I={w.I} N={w.N} tokens "
+                        f"({w.meta.get('n_visual', '?')} visual + text per sequence), kept={w.n_kept}",
+            "C": w.C, "I": w.I, "tokens": w.N, "kept_tokens": w.n_kept, "skip_ratio": args.skip_ratio,
+            "l2_policy": "inputs larger than L2 (weights 3 x %.0f MB re-read every step)" % (w.C * w.I * 2 / 1e6),
+            "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2503_21817_b200 as sk
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    w = make_workload(args, rank)
+    N, C, I, nk = w.N, w.C, w.I, w.n_kept
+
+    def h_bf16(a):
+        return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).reshape(a.shape)
+
+    # pinned host copies of the step's inputs and results (for the end-to-end leg)
+    hx, hdout = h_bf16(w.x).pin_memory(), h_bf16(w.dout).pin_memory()
+    hmask = torch.from_numpy(w.skip_mask).pin_memory()
+    hout, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    x, dout, mask = hx.to(dev), hdout.to(dev), hmask.to(dev)
+    Wg, Wu, Wd = h_bf16(w.W_gate).to(dev), h_bf16(w.W_up).to(dev), h_bf16(w.W_down).to(dev)
+    out, dx = torch.empty_like(x), torch.empty_like(x)
+    dWg, dWu, dWd = torch.empty_like(Wg), torch.empty_like(Wu), torch.empty_like(Wd)
+    ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense)
+    if args.dense:
+        nk = N
+
+    def step():
+        ctx.forward(x, mask, Wg, Wu, Wd, out=out)
+        ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+
+    def step_e2e():
+        x.copy_(hx, non_blocking=True)
+        mask.copy_(hmask, non_blocking=True)
+        dout.copy_(hdout, non_blocking=True)
+        step()
+        hout.copy_(out, non_blocking=True)
+        hdx.copy_(dx, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0 = time.time()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        t1 = time.time()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, t0, t1
+
+    if args.profile_only:      # short launch sequence for ncu: W + K steps, nothing else
+        for _ in range(args.warmup + args.steps):
+            step()
+        ctx.poll()
+        print(json.dumps({"profile_only": True, "launches_per_step": sum(ctx.launches())}), flush=True)
+        return
+    for _ in range(max(args.warmup, 3)):
+        step()
+    ctx.poll()
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms, t0, t1 = timed(step, args.steps)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    ctx.poll()
+    launches_per_step = sum(ctx.launches())
+
+    for _ in range(2):
+        step_e2e()
+    ms_e2e, _, _ = timed(step_e2e, args.steps)
+
+    # per-kernel durations: the same steps again with CUDA events recorded around every launch
+    prof = ctx.profile(step, args.steps) if hasattr(ctx, "profile") else None
+    ctx.poll()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    ms_step = ms / args.steps
+    flops = sk.skipffn_flops(C, I, nk)
+    value = world * nk / (ms_step * 1e-3)
+    tflops = world * flops / (ms_step * 1e-3) / 1e12
+    unit_flops = 2.0 * nk * C * I     # one GEMM "unit" of the path: 2 * Nk * C * I
+    kernel_units = {"gateup": 2, "down": 1, "dh": 1, "dw_down": 1, "dw_gate": 1, "dw_up": 1, "dx": 2}
+    kernels, roofline = {}, None
+    if prof:
+        total = sum(prof.values())
+        for name, kms in prof.items():
+            ent = {"ms": kms, "share": kms / total if total else None}
+            if name in kernel_units:
+                ent["tflops"] = kernel_units[name] * unit_flops / (kms * 1e-3) / 1e12
+                ent["frac_of_measured_bf16_peak"] = ent["tflops"] / pk["bf16_tflops"]
+            kernels[name] = ent
+        gemms = {k: v for k, v in kernels.items() if k in kernel_units}
+        top = max(gemms, key=lambda k: gemms[k]["ms"])
+        roofline = {"kernel": f"k_umma_gemm[{top}]", "bound": "tensor", "achieved": gemms[top]["tflops"],
+                    "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemms[top]["tflops"] / pk["bf16_tflops"],
+                    "peak_source": pk["source"] + " (burst cuBLAS bf16)",
+                    "traffic": NCU_TRAFFIC_BYTES.get(top),
+                    "all_gemm_kernels": {"tflops": sum(kernel_units.values()) * unit_flops /
+                                         (sum(v["ms"] for v in gemms.values()) * 1e-3) / 1e12}}
+        roofline["all_gemm_kernels"]["frac"] = roofline["all_gemm_kernels"]["tflops"] / pk["bf16_tflops"]
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        rate, kept, dt, cores = oracle_sample_rate(w, args.cpu_sample_tokens)
+        cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {args.cpu_sample_tokens} tokens of sequence 0 ({kept} kept), full fp64 "
+                         f"forward+backward, {dt:.1f} s"}
+
+    h2d = hx.numel() * 2 + hdout.numel() * 2 + hmask.numel()
+    d2h = hout.numel() * 2 + hdx.numel() * 2
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(args, w), "tflops": tflops,
+            "frac_of_measured_bf16_peak": tflops / world / pk["bf16_tflops"],
+            "frac_of_sustained_bf16_peak": (tflops / world / pk["bf16_tflops_sustained"]) if pk["bf16_tflops_sustained"] else None,
+            "frac_of_nominal_bf16_peak": tflops / world / 2250.0,
+            "e2e": {"value": world * nk / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
+            "kernels": kernels, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--shape", default="llama3-8b", choices=list(wl.SWEEP_SHAPES))
+    ap.add_argument("--skip-ratio", type=float, default=0.75)
+    ap.add_argument("--dense", action="store_true", help="in-library dense comparator (mask ignored)")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--cpu-sample-tokens", type=int, default=24)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile-only", action="store_true",
+                    help="run warmup+steps steps and exit (launch sequence for an ncu capture)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

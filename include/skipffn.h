@@ -113,6 +113,16 @@ skipffn_status skipffn_get_intermediate(const skipffn_saved *saved, int32_t whic
  * stream reports an error, else SKIPFFN_OK.  The word is cleared. */
 skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_out);
 
+/* Per-launch timing for benchmarks.  While enabled, forward / backward record a CUDA event on the
+ * caller's stream before and after each kernel launch (no synchronisation).  skipffn_profile_read
+ * waits for those events and writes the elapsed milliseconds of each launch slot into
+ * ms[SKIPFFN_PROFILE_SLOTS] (0 for slots that did not run): 0 mask compaction, 1 routing of x,
+ * 2 gate/up GEMM, 3 down GEMM, 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate, 8 dW_up,
+ * 9 dX GEMM. */
+#define SKIPFFN_PROFILE_SLOTS 10
+skipffn_status skipffn_profile_enable(skipffn_saved *saved, int32_t on);
+skipffn_status skipffn_profile_read(skipffn_saved *saved, float *ms);
+
 /* Number of kernels the last forward (which=0) or backward (which=1) call enqueued. */
 int32_t skipffn_last_launches(const skipffn_saved *saved, int32_t which);
 

@@ -16,7 +16,10 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_destroy",
            "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
-           "skipffn_strerror"]
+           "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read"]
+
+PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
+                 "dw_up", "dx"]
 
 
 class SkipFFNError(RuntimeError):
@@ -65,6 +68,10 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_last_launches.argtypes = [vp, i32]
     lib.skipffn_flops.restype = ctypes.c_double
     lib.skipffn_flops.argtypes = [cfgp, i64]
+    lib.skipffn_profile_enable.restype = i32
+    lib.skipffn_profile_enable.argtypes = [vp, i32]
+    lib.skipffn_profile_read.restype = i32
+    lib.skipffn_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -248,6 +255,26 @@ class SkipFFN:
         off = ptr - self.workspace.data_ptr()
         nbytes = numel * torch.empty(0, dtype=dtype).element_size()
         return self.workspace[off:off + nbytes].view(dtype)
+
+    def profile(self, step_fn, steps: int):
+        """Run ``step_fn`` ``steps`` times with CUDA events around every kernel launch; returns the
+        mean milliseconds per launch slot (``PROFILE_SLOTS`` names)."""
+        st = self.lib.skipffn_profile_enable(self._saved, 1)
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_profile_enable")
+        acc = [0.0] * len(PROFILE_SLOTS)
+        buf = (ctypes.c_float * len(PROFILE_SLOTS))()
+        try:
+            for _ in range(steps):
+                step_fn()
+                st = self.lib.skipffn_profile_read(self._saved, buf)
+                if st != 0:
+                    raise SkipFFNError(st, "skipffn_profile_read")
+                for i in range(len(PROFILE_SLOTS)):
+                    acc[i] += buf[i]
+        finally:
+            self.lib.skipffn_profile_enable(self._saved, 0)
+        return {n: a / steps for n, a in zip(PROFILE_SLOTS, acc) if a > 0}
 
     def launches(self):
         return (int(self.lib.skipffn_last_launches(self._saved, 0)),

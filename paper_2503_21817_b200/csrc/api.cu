@@ -19,6 +19,10 @@ struct skipffn_saved {
     int forwarded;
     const void *Wg, *Wu, *Wd;
     int launches[2];
+    // optional per-launch timing (CUDA events on the caller's stream)
+    int profiling;
+    cudaEvent_t ev[2 * SKIPFFN_PROFILE_SLOTS];
+    int ev_recorded[SKIPFFN_PROFILE_SLOTS];
 };
 
 namespace {
@@ -61,10 +65,30 @@ bool use_umma(const skipffn_saved *s)
     return s->cfg.dtype == SKIPFFN_BF16 && s->cfg.path == SKIPFFN_PATH_DEFAULT;
 }
 
-cudaError_t run_gemm(skipffn_saved *s, int which, int epi, const GemmArgs &g, cudaStream_t st)
+// Launch slots (also the order of skipffn_profile_read): forward 0 compaction, 1 routing of x,
+// 2 gate/up GEMM, 3 down GEMM; backward 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate,
+// 8 dW_up, 9 dX GEMM.
+enum : int { SLOT_COMPACT = 0, SLOT_ROUTE_X, SLOT_GATEUP, SLOT_DOWN, SLOT_ROUTE_DOUT, SLOT_DH,
+             SLOT_DW_DOWN, SLOT_DW_GATE, SLOT_DW_UP, SLOT_DX };
+
+template <typename F>
+cudaError_t timed_launch(skipffn_saved *s, int slot, cudaStream_t st, F &&launch)
 {
-    s->launches[which]++;
-    return use_umma(s) ? launch_umma_gemm(epi, g, st) : launch_simt_gemm(epi, s->cfg.dtype, g, st);
+    s->launches[slot >= SLOT_ROUTE_DOUT ? 1 : 0]++;
+    if (!s->profiling) return launch();
+    cudaError_t e = cudaEventRecord(s->ev[2 * slot], st);
+    if (e != cudaSuccess) return e;
+    e = launch();
+    if (e != cudaSuccess) return e;
+    s->ev_recorded[slot] = 1;
+    return cudaEventRecord(s->ev[2 * slot + 1], st);
+}
+
+cudaError_t run_gemm(skipffn_saved *s, int slot, int epi, const GemmArgs &g, cudaStream_t st)
+{
+    return timed_launch(s, slot, st, [&] {
+        return use_umma(s) ? launch_umma_gemm(epi, g, st) : launch_simt_gemm(epi, s->cfg.dtype, g, st);
+    });
 }
 
 GemmArgs base_args(const skipffn_saved *s)
@@ -78,9 +102,11 @@ GemmArgs base_args(const skipffn_saved *s)
 
 skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int which, cudaStream_t st)
 {
+    (void)which;
     if (N > 0) {
-        s->launches[which]++;
-        if (launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, st) != cudaSuccess)
+        if (timed_launch(s, SLOT_COMPACT, st, [&] {
+                return launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, st);
+            }) != cudaSuccess)
             return SKIPFFN_ECUDA;
     } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
         return SKIPFFN_ECUDA;
@@ -129,7 +155,44 @@ skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config 
     return SKIPFFN_OK;
 }
 
-void skipffn_saved_destroy(skipffn_saved *saved) { delete saved; }
+void skipffn_saved_destroy(skipffn_saved *saved)
+{
+    if (!saved) return;
+    if (saved->profiling)
+        for (int i = 0; i < 2 * SKIPFFN_PROFILE_SLOTS; ++i) cudaEventDestroy(saved->ev[i]);
+    delete saved;
+}
+
+skipffn_status skipffn_profile_enable(skipffn_saved *s, int32_t on)
+{
+    if (!s) return SKIPFFN_EINVAL;
+    if (on && !s->profiling) {
+        for (int i = 0; i < 2 * SKIPFFN_PROFILE_SLOTS; ++i)
+            if (cudaEventCreate(&s->ev[i]) != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(s->ev[j]);
+                return SKIPFFN_ECUDA;
+            }
+        s->profiling = 1;
+    } else if (!on && s->profiling) {
+        for (int i = 0; i < 2 * SKIPFFN_PROFILE_SLOTS; ++i) cudaEventDestroy(s->ev[i]);
+        s->profiling = 0;
+    }
+    memset(s->ev_recorded, 0, sizeof(s->ev_recorded));
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_profile_read(skipffn_saved *s, float *ms)
+{
+    if (!s || !ms || !s->profiling) return SKIPFFN_EINVAL;
+    for (int i = 0; i < SKIPFFN_PROFILE_SLOTS; ++i) {
+        ms[i] = 0.0f;
+        if (!s->ev_recorded[i]) continue;
+        if (cudaEventSynchronize(s->ev[2 * i + 1]) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (cudaEventElapsedTime(&ms[i], s->ev[2 * i], s->ev[2 * i + 1]) != cudaSuccess) return SKIPFFN_ECUDA;
+        s->ev_recorded[i] = 0;
+    }
+    return SKIPFFN_OK;
+}
 
 skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t N, void *stream)
 {
@@ -163,7 +226,7 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     cudaStream_t st = (cudaStream_t)stream;
     const int C = s->cfg.C, I = s->cfg.I;
     s->forwarded = 0;
-    if (skip_mask || s->cfg.dense) {
+    if (skip_mask || s->cfg.dense || N == 0) {
         if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, ST_WORDS * 4, st) != cudaSuccess)
             return SKIPFFN_ECUDA;
         s->launches[0] = 0;
@@ -180,8 +243,8 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     RouteArgs r;
     r.src = x; r.dst_compact = s->Xk; r.dst_identity = out; r.pos = s->pos; r.status = s->status;
     r.N = N; r.C = C; r.elem_bytes = s->esize;
-    s->launches[0]++;
-    if (launch_route(r, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (timed_launch(s, SLOT_ROUTE_X, st, [&] { return launch_route(r, st); }) != cudaSuccess)
+        return SKIPFFN_ECUDA;
 
     // G = Xk Wg^T, U = Xk Wu^T, H = silu(G) * U
     GemmArgs g = base_args(s);
@@ -189,7 +252,7 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
     g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
     g.out0 = s->G; g.out1 = s->U; g.out2 = s->H; g.ldo = I;
-    if (run_gemm(s, 0, EPI_GATEUP, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (run_gemm(s, SLOT_GATEUP, EPI_GATEUP, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
 
     // out[idx[r]] = Xk[r] + H Wd^T
     g = base_args(s);
@@ -197,7 +260,7 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     g.B = W_down; g.ldb_n = I; g.ldb_k = 1; g.b_outer = C;
     g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
     g.in0 = s->Xk; g.out0 = out; g.ldo = C;
-    if (run_gemm(s, 0, EPI_DOWN, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (run_gemm(s, SLOT_DOWN, EPI_DOWN, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     s->forwarded = 1;
     return SKIPFFN_OK;
 }
@@ -219,8 +282,8 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         RouteArgs r;
         r.src = dout; r.dst_compact = s->dOk; r.dst_identity = dx; r.pos = s->pos; r.status = s->status;
         r.N = N; r.C = C; r.elem_bytes = s->esize;
-        s->launches[1]++;
-        if (launch_route(r, st) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (timed_launch(s, SLOT_ROUTE_DOUT, st, [&] { return launch_route(r, st); }) != cudaSuccess)
+            return SKIPFFN_ECUDA;
 
         // dH = dOk Wd ; dG, dU through the activation
         g = base_args(s);
@@ -228,7 +291,7 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;
         g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
         g.in0 = s->G; g.in1 = s->U; g.out0 = s->dG; g.out1 = s->dU; g.ldo = I;
-        if (run_gemm(s, 1, EPI_DH, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (run_gemm(s, SLOT_DH, EPI_DH, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
         return SKIPFFN_ECUDA;
     }
@@ -241,7 +304,7 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         g.B = s->H; g.ldb_n = 1; g.ldb_k = I; g.b_outer = s->cap;
         g.M = C; g.N = I; g.K = kmax; g.k_from_nk = 1;
         g.out0 = dW_down; g.ldo = I; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
-        if (run_gemm(s, 1, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (run_gemm(s, SLOT_DW_DOWN, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     }
     for (int w = 0; w < 2; ++w) {   // dWg[i, c] = sum_r dG[r, i] Xk[r, c]; same for up with dU
         void *dst = w == 0 ? dW_gate : dW_up;
@@ -251,7 +314,7 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         g.B = s->Xk; g.ldb_n = 1; g.ldb_k = C; g.b_outer = s->cap;
         g.M = I; g.N = C; g.K = kmax; g.k_from_nk = 1;
         g.out0 = dst; g.ldo = C; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
-        if (run_gemm(s, 1, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (run_gemm(s, w == 0 ? SLOT_DW_GATE : SLOT_DW_UP, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     }
 
     if (N > 0) {   // dx[idx[r]] = dOk[r] + dG Wg + dU Wu
@@ -260,7 +323,7 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
         g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
         g.in0 = s->dOk; g.out0 = dx; g.ldo = C;
-        if (run_gemm(s, 1, EPI_DX, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+        if (run_gemm(s, SLOT_DX, EPI_DX, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     }
     return SKIPFFN_OK;
 }

@@ -1,0 +1,294 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the
+same seeded inputs.  Index lists and identity rows bit-exact; floating point within the stated
+tolerances (tests/parity.py)."""
+import ctypes
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+from gpu_util import DeviceWorkload, bits, run, to_dev, to_host
+from parity import check, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+
+def _sk():
+    import paper_2503_21817_b200 as sk
+    return sk
+
+
+def _oracle_all(w, mask=None):
+    m = w.skip_mask if mask is None else mask
+    out = oracle.forward(w.x, m, w.W_gate, w.W_up, w.W_down)
+    dx, dwg, dwu, dwd = oracle.backward(w.x, m, w.W_gate, w.W_up, w.W_down, w.dout)
+    return dict(out=out, dx=dx, dW_gate=dwg, dW_up=dwu, dW_down=dwd)
+
+
+def _compare(w, r, ref, mask=None):
+    m = w.skip_mask if mask is None else mask
+    N, C = w.N, w.C
+    out = r["out"].reshape(N, C)
+    dx = r["dx"].reshape(N, C)
+    kept = m == 0
+    # integer / byte work: index list and identity rows are bit-exact
+    idx, nk = r["ctx"].kept()
+    assert nk == int(kept.sum())
+    assert np.array_equal(idx.cpu().numpy(), oracle.compact(m))
+    xb, db = bits(r["dev"].x.reshape(N, C)), bits(r["dev"].dout.reshape(N, C))
+    assert np.array_equal(bits(out)[~kept], xb[~kept])
+    assert np.array_equal(bits(dx)[~kept], db[~kept])
+    # floating point
+    check(to_host(out), ref["out"], w.dtype, "out")
+    check(to_host(dx), ref["dx"], w.dtype, "dx")
+    for k in ("dW_gate", "dW_up", "dW_down"):
+        if kept.any():
+            check(to_host(r[k]), ref[k], w.dtype, k, few_terms=int(kept.sum()) < 8)
+        else:
+            assert not to_host(r[k]).any()
+    # the FFN branch alone (out - x on kept rows), so that the O(1) residual cannot hide an FFN
+    # error: its error budget is the tolerance on FFN(x) plus the rounding of `out` itself
+    if kept.any():
+        x64 = w.x.astype(np.float64)
+        ffn_ref = (ref["out"] - x64)[kept]
+        ffn_got = (to_host(out) - x64)[kept]
+        eps_out = 2.0 ** -9 if w.dtype == "bf16" else 2.0 ** -24
+        tol = (5e-3 if w.dtype == "bf16" else 1e-5) * np.linalg.norm(ffn_ref) + \
+            eps_out * np.linalg.norm(ref["out"][kept])
+        assert np.linalg.norm(ffn_got - ffn_ref) <= tol
+
+
+# ------------------------------------------------------------------ a1: compaction
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 1000, 4928, 16384, 16385, 50001])
+def test_compaction_bit_exact(N):
+    import torch
+    sk = _sk()
+    r = np.random.default_rng(N)
+    m = ((r.random(N) < 0.7) * r.integers(1, 256, size=N)).astype(np.uint8)
+    for mask in (m, np.zeros(N, np.uint8), np.full(N, 255, np.uint8)):
+        ctx = sk.SkipFFN(64, 64, N)
+        ctx.plan(torch.from_numpy(mask).cuda())
+        idx, nk = ctx.kept()
+        ref = oracle.compact(mask)
+        assert nk == ref.size == N - np.count_nonzero(mask)
+        assert np.array_equal(idx.cpu().numpy(), ref)
+    dense = sk.SkipFFN(64, 64, N, dense=True)
+    dense.plan(torch.from_numpy(m).cuda())
+    idx, nk = dense.kept()
+    assert nk == N and np.array_equal(idx.cpu().numpy(), np.arange(N))
+
+
+# ------------------------------------------------------------------ configs[0]
+@pytest.mark.parametrize("dtype,path", [("fp32", 0), ("bf16", 0), ("bf16", 1)])
+def test_config1_tiny(dtype, path):
+    w = wl.config1(dtype=dtype)
+    _compare(w, run(w, path=path), _oracle_all(w))
+
+
+# ------------------------------------------------------------------ several tiles + ragged tails
+@pytest.mark.parametrize("dtype,path", [("bf16", 0), ("fp32", 0), ("bf16", 1)])
+def test_multi_tile_ragged(dtype, path):
+    # C = 576 (2.25 N-tiles of 256, 9 K-blocks), I = 1000 (ragged N and K), Nk = 300 (2.3 M-tiles)
+    w = wl.small_case(1, dtype, 576, 1000, 3, 20, 200, 0.6)
+    assert w.n_kept == 300
+    _compare(w, run(w, path=path), _oracle_all(w))
+
+
+def test_contiguous_span_layout():
+    # the paper's layout: one contiguous skipped span per sequence
+    w = wl.uniform_batch(2, "bf16", 256, 512, 4, 10, 150, 10, skip_ratio=0.8, contiguous_span=True)
+    _compare(w, run(w), _oracle_all(w))
+
+
+def test_packed_variable_length_small():
+    w = wl.config4(seed=3, C=128, I=256, n_seq=3)
+    _compare(w, run(w), _oracle_all(w))
+    # bad offsets are rejected on the host
+    sk = _sk()
+    dev = DeviceWorkload(w)
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    bad = w.cu_seqlens.copy()
+    bad[-1] -= 1
+    with pytest.raises(sk.SkipFFNError):
+        ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down, cu_seqlens=bad)
+
+
+# ------------------------------------------------------------------ degenerate kept counts
+@pytest.mark.parametrize("nk", [0, 1, 127, 128, 129, 257])
+def test_kept_count_edges(nk):
+    base = wl.uniform_batch(5, "bf16", 128, 256, 1, 0, 300, 0, n_skip=300 - nk)
+    assert base.n_kept == nk
+    r = run(base)
+    _compare(base, r, _oracle_all(base))
+    if nk == 0:   # all skipped: out == x, dx == dout bitwise, zero weight gradients
+        assert np.array_equal(bits(r["out"]), bits(r["dev"].x))
+        assert np.array_equal(bits(r["dx"]), bits(r["dev"].dout))
+
+
+def test_empty_batch():
+    import torch
+    sk = _sk()
+    ctx = sk.SkipFFN(128, 256, 16)
+    w = wl.uniform_batch(0, "bf16", 128, 256, 1, 0, 4, 0, n_skip=0)
+    dev = DeviceWorkload(w)
+    x = torch.empty(0, 128, dtype=torch.bfloat16, device="cuda")
+    out = ctx.forward(x, torch.empty(0, dtype=torch.uint8, device="cuda"), dev.W_gate, dev.W_up, dev.W_down)
+    dx, dwg, dwu, dwd = ctx.backward(torch.empty_like(x))
+    ctx.poll()
+    assert out.numel() == 0 and dx.numel() == 0
+    assert not dwg.float().any() and not dwu.float().any() and not dwd.float().any()
+
+
+# ------------------------------------------------------------------ all kept == dense comparator
+def test_all_kept_equals_dense_and_eq8_skip_error():
+    w = wl.small_case(7, "bf16", 256, 512, 2, 16, 120, 0.5)
+    zeros = np.zeros_like(w.skip_mask)
+    ref_dense = _oracle_all(w, zeros)
+    w_all = wl.small_case(7, "bf16", 256, 512, 2, 16, 120, 0.0)
+    assert np.array_equal(w_all.x, w.x) and not w_all.skip_mask.any()
+    r_all = run(w_all)
+    r_dense = run(w, dense=True)          # mask present but ignored
+    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+        assert np.array_equal(bits(r_all[k]), bits(r_dense[k])), k
+    _compare(w, r_dense, ref_dense, zeros)
+    # Eq. 8: on a skipped row the dense output differs from the skip output by FFN(x)
+    r_skip = run(w)
+    sk_rows = w.skip_mask != 0
+    diff = (to_host(r_dense["out"]) - to_host(r_skip["out"])).reshape(w.N, w.C)[sk_rows]
+    ffn = oracle.forward(w.x, zeros, w.W_gate, w.W_up, w.W_down, ffn_only=True)[sk_rows]
+    x_norm = np.linalg.norm(w.x[sk_rows])
+    assert np.linalg.norm(diff - ffn) <= 5e-3 * np.linalg.norm(ffn) + 2.0 ** -9 * x_norm
+
+
+# ------------------------------------------------------------------ aliasing, poisoning, options
+def test_inplace_aliasing_matches_out_of_place():
+    w = wl.small_case(9, "bf16", 256, 512, 2, 16, 120, 0.7)
+    a = run(w)
+    b = run(w, inplace=True)
+    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+        assert np.array_equal(bits(a[k]), bits(b[k])), k
+
+
+def test_poisoned_skipped_rows_do_not_leak():
+    import torch
+    w = wl.small_case(11, "bf16", 256, 512, 2, 16, 120, 0.7)
+    clean = run(w)
+    dev = DeviceWorkload(w)
+    sk_rows = torch.from_numpy(w.skip_mask != 0).cuda()
+    dev.x[sk_rows] = float("nan")
+    dev.dout[sk_rows] = float("inf")
+    dirty = run(w, dev=dev)
+    kept = w.skip_mask == 0
+    N, C = w.N, w.C
+    assert np.array_equal(bits(clean["out"].reshape(N, C))[kept], bits(dirty["out"].reshape(N, C))[kept])
+    assert np.array_equal(bits(clean["dx"].reshape(N, C))[kept], bits(dirty["dx"].reshape(N, C))[kept])
+    for k in ("dW_gate", "dW_up", "dW_down"):
+        assert np.array_equal(bits(clean[k]), bits(dirty[k])), k
+    # the poisoned rows themselves pass through bit-exactly (NaN payloads included)
+    assert np.array_equal(bits(dirty["out"].reshape(N, C))[~kept], bits(dev.x.reshape(N, C))[~kept])
+
+
+@pytest.mark.parametrize("path", [0, 1])
+def test_fp32_gradients_and_accumulation(path):
+    import torch
+    w = wl.small_case(13, "bf16", 256, 512, 2, 16, 120, 0.7)
+    ref = _oracle_all(w)
+    r = run(w, grad_fp32=True, path=path)
+    assert r["dW_gate"].dtype == torch.float32
+    _compare(w, r, ref)
+    # fp32 gradients carry no output rounding: tighter than the bf16 bound
+    assert rel_fro(to_host(r["dW_down"]), ref["dW_down"]) < 4e-3
+    init = [torch.full((w.I, w.C), 0.5, device="cuda"), torch.full((w.I, w.C), -0.25, device="cuda"),
+            torch.full((w.C, w.I), 1.0, device="cuda")]
+    r2 = run(w, grad_fp32=True, accumulate_dw=True, dw_init=[t.clone() for t in init], path=path)
+    for k, t in zip(("dW_gate", "dW_up", "dW_down"), init):
+        assert torch.equal(r2[k], r[k] + t), k
+
+
+def test_plan_once_reuse_for_next_layer():
+    sk = _sk()
+    w = wl.small_case(15, "bf16", 256, 512, 2, 16, 120, 0.7)
+    dev = DeviceWorkload(w)
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    ctx.plan(dev.mask)
+    out1 = ctx.forward(dev.x, None, dev.W_gate, dev.W_up, dev.W_down)       # reuses the list
+    out2 = ctx.forward(out1, None, dev.W_up, dev.W_gate, dev.W_down)        # "next layer"
+    ctx.poll()
+    ref1 = oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down)
+    check(to_host(out1), ref1, "bf16", "layer 1")
+    ref2 = oracle.forward(to_host(out1), w.skip_mask, w.W_up, w.W_gate, w.W_down)
+    check(to_host(out2), ref2, "bf16", "layer 2")
+    # without a list to reuse the call is rejected
+    fresh = sk.SkipFFN(w.C, w.I, w.N)
+    with pytest.raises(sk.SkipFFNError):
+        fresh.forward(dev.x, None, dev.W_gate, dev.W_up, dev.W_down)
+
+
+def test_run_twice_bit_identical():
+    w = wl.small_case(17, "bf16", 576, 1000, 3, 20, 200, 0.6)
+    a, b = run(w), run(w)
+    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+        assert np.array_equal(bits(a[k]), bits(b[k])), k
+
+
+def test_unsupported_and_invalid_arguments():
+    import torch
+    sk = _sk()
+    with pytest.raises(sk.SkipFFNError):
+        sk.SkipFFN(100, 256, 16)                       # C % 8 != 0
+    ctx = sk.SkipFFN(128, 256, 16)
+    w = wl.uniform_batch(0, "bf16", 128, 256, 1, 0, 32, 0, n_skip=8)
+    dev = DeviceWorkload(w)
+    with pytest.raises(sk.SkipFFNError):
+        ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)   # 32 tokens > max_tokens 16
+    with pytest.raises(sk.SkipFFNError):
+        ctx.backward(dev.dout)                                               # no forward yet
+
+
+# ------------------------------------------------------------------ full size, sampled oracle
+def _sampled_full_size(w, n_tok=10, n_col=6, dense=False):
+    """Full-size run in the benchmark's launch configuration; the oracle computes sampled output
+    rows and sampled weight-gradient rows / columns one by one."""
+    r = run(w, dense=dense)
+    m = np.zeros_like(w.skip_mask) if dense else w.skip_mask
+    N, C = w.N, w.C
+    rng = np.random.default_rng(0)
+    kept_tok = np.flatnonzero(m == 0)
+    skip_tok = np.flatnonzero(m != 0)
+    tok = np.concatenate([rng.choice(kept_tok, n_tok, replace=False),
+                          [kept_tok[0], kept_tok[-1]],
+                          rng.choice(skip_tok, 3, replace=False) if skip_tok.size else []]).astype(np.int64)
+    cols = np.concatenate([rng.choice(w.I, n_col, replace=False), [0, w.I - 1]]).astype(np.int64)
+    x64, wg, wu, wd, do = (a.astype(np.float64) for a in (w.x, w.W_gate, w.W_up, w.W_down, w.dout))
+    out_r, dx_r = oracle.rows(x64, m, wg, wu, wd, do, tok)
+    a, b, c = oracle.dw_columns(x64, m, wg, wu, wd, do, cols)
+    out = to_host(r["out"].reshape(N, C)[tok])
+    dx = to_host(r["dx"].reshape(N, C)[tok])
+    check(out, out_r, "bf16", "out rows")
+    check(dx, dx_r, "bf16", "dx rows")
+    check(to_host(r["dW_gate"][cols]), a, "bf16", "dW_gate rows")
+    check(to_host(r["dW_up"][cols]), b, "bf16", "dW_up rows")
+    check(to_host(r["dW_down"][:, cols].T), c, "bf16", "dW_down cols")
+    # properties that hold at any size: exact index list, identity rows, finite everywhere
+    idx, nk = r["ctx"].kept()
+    assert np.array_equal(idx.cpu().numpy(), oracle.compact(m))
+    kept = m == 0
+    assert np.array_equal(bits(r["out"].reshape(N, C))[~kept], bits(r["dev"].x.reshape(N, C))[~kept])
+    assert np.array_equal(bits(r["dx"].reshape(N, C))[~kept], bits(r["dev"].dout.reshape(N, C))[~kept])
+    import torch
+    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+        assert bool(torch.isfinite(r[k].float()).all()), k
+    return r
+
+
+def test_config2_llama3_8b_full_size_sampled():
+    w = wl.config2()
+    assert (w.N, w.n_kept, w.C, w.I) == (4928, 1472, 4096, 14336)
+    _sampled_full_size(w)
+
+
+def test_config3_highres_full_size_sampled():
+    w = wl.config3()
+    assert (w.N, w.n_kept) == (9376, 1312)
+    _sampled_full_size(w, n_tok=6, n_col=4)
