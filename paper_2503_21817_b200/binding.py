@@ -133,6 +133,7 @@ class SkipFFN:
         if st != 0:
             raise SkipFFNError(st, "skipffn_saved_create")
         self._keep = []   # tensors the handle borrows between forward and backward
+        self._shape = None
 
     def __del__(self):
         if getattr(self, "_saved", None) and self._saved.value:
@@ -201,6 +202,8 @@ class SkipFFN:
 
     def backward(self, dout, dx=None, dW_gate=None, dW_up=None, dW_down=None, need_dw=True):
         torch, dt = self._torch, self.torch_dtype
+        if self._shape is None:
+            raise SkipFFNError(1, "skipffn_backward (no forward has run on this context)")
         self._check(dout, "dout", self._shape, dt)
         if dx is None:
             dx = torch.empty_like(dout)

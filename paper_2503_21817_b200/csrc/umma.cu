@@ -20,6 +20,7 @@
 // host synchronisation sits between mask compaction and the GEMMs.  Every mbarrier wait is
 // bounded: on expiry the CTA records SKIPFFN_ETIMEOUT plus a site code and leaves normally.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -33,8 +34,11 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KiB
 constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64-wide MN-major slab of BK rows: 8 KiB
 constexpr int ACC_COLS = 256;                    // fp32 columns per accumulator
 constexpr int TMEM_COLS = 512;
-constexpr int UMMA_THREADS = 192;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int EPI_WARPS = 8;
+constexpr int EPI_BUF_BYTES = 2048;              // per-warp staging: 32 rows x 64 B
+constexpr int UMMA_THREADS = 64 + 32 * EPI_WARPS;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES + 1024 /*alignment slack*/ +
+                           256 /*barriers*/;
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s
 
 // ------------------------------------------------------------------------------------ PTX
@@ -180,11 +184,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 256.
-__host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major)
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n (a multiple of 16, at most 256).
+__host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major, int n)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) |
-           ((uint32_t)b_mn_major << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -192,6 +196,7 @@ struct UmmaParams {
     int32_t M, N, K;                 // host upper bounds
     int32_t m_from_nk, k_from_nk;    // extent is the device-resident kept count
     int32_t segments;                // 2: second K segment reads tmA2 / tmB2 (dX)
+    int32_t force_bn;                // > 0: tile width override (tuning)
     int32_t *status;
     const int32_t *idx;
     void *out0, *out1, *out2;
@@ -218,6 +223,96 @@ __device__ __forceinline__ void unpack_bf16(uint32_t w, float &lo, float &hi)
     hi = __high2float(v);
 }
 
+// sigmoid from the hardware exp2 / reciprocal approximations (relative error ~1e-6, far below the
+// bf16 rounding of everything it feeds)
+__device__ __forceinline__ float fast_sigmoid(float z) { return __fdividef(1.0f, 1.0f + __expf(-z)); }
+__device__ __forceinline__ float fast_swiglu(float g, float u) { return g * fast_sigmoid(g) * u; }
+__device__ __forceinline__ void fast_swiglu_bwd(float dh, float g, float u, float &dg, float &du)
+{
+    float s = fast_sigmoid(g);
+    du = dh * (g * s);
+    dg = dh * u * (s * (1.0f + g * (1.0f - s)));
+}
+
+// Tile width (accumulator columns) for this launch.  With few M tiles the tile count rarely fills
+// a whole number of waves of the persistent grid; narrower tiles trade MMA width for fewer idle
+// SMs in the last wave.  Cost model: waves x (MMA columns + B columns loaded, in 64-wide slabs).
+__device__ __forceinline__ int choose_bn(int num_m, int N, int grid, int force_bn)
+{
+    if (force_bn > 0) return force_bn;
+    int best = BN;
+    long best_cost = -1;
+    for (int bn = BN; bn >= 128; bn -= 16) {
+        const int num_n = (N + bn - 1) / bn;
+        const long tiles = (long)num_m * num_n;
+        const long waves = (tiles + grid - 1) / grid;
+        const long cost = waves * (bn + 64 * ((bn + 63) / 64) + 32);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+// Epilogue staging.  A warp owns 32 accumulator rows (one per lane).  For a 32-column bf16 chunk
+// each lane holds its row as 16 packed words (64 B).  The rows are written to a 2 KiB per-warp
+// shared-memory buffer (16-byte slots XOR-swizzled by row pair: conflict-free both ways), then read
+// back so that four consecutive lanes cover one row's 64 contiguous bytes: every global store
+// instruction writes eight full 64-byte row segments instead of 32 scattered 16-byte pieces.
+// `my_row` is this lane's destination (row pointer at the chunk's first column) or null for a row
+// that must not be written; `valid_slots` = number of 16-byte slots inside the column range.
+__device__ __forceinline__ void store_rows_64B(uint32_t sbuf, int lane, const uint32_t (&w)[16],
+                                               char *my_row, int valid_slots)
+{
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + lane * 64 + ((c ^ sw) << 4)),
+                     "r"(w[4 * c]), "r"(w[4 * c + 1]), "r"(w[4 * c + 2]), "r"(w[4 * c + 3])
+                     : "memory");
+    __syncwarp();
+    const int c = lane & 3;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = it * 8 + (lane >> 2);
+        uint4 v;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                     : "r"(sbuf + row * 64 + ((c ^ ((row >> 1) & 3)) << 4))
+                     : "memory");
+        char *dst = (char *)__shfl_sync(0xffffffffu, (unsigned long long)my_row, row);
+        if (dst != nullptr && c < valid_slots) *reinterpret_cast<uint4 *>(dst + c * 16) = v;
+    }
+    __syncwarp();
+}
+// fp32 variant with read-modify-write (dW accumulation): same staging, 16 columns per call
+__device__ __forceinline__ void store_rows_64B_f32(uint32_t sbuf, int lane, const uint32_t (&w)[16],
+                                                   char *my_row, int valid_slots, int accumulate)
+{
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + lane * 64 + ((c ^ sw) << 4)),
+                     "r"(w[4 * c]), "r"(w[4 * c + 1]), "r"(w[4 * c + 2]), "r"(w[4 * c + 3])
+                     : "memory");
+    __syncwarp();
+    const int c = lane & 3;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = it * 8 + (lane >> 2);
+        float4 v;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                     : "r"(sbuf + row * 64 + ((c ^ ((row >> 1) & 3)) << 4))
+                     : "memory");
+        char *dst = (char *)__shfl_sync(0xffffffffu, (unsigned long long)my_row, row);
+        if (dst != nullptr && c < valid_slots) {
+            float4 *d = reinterpret_cast<float4 *>(dst + c * 16);
+            if (accumulate) { float4 o = *d; v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w; }
+            *d = v;
+        }
+    }
+    __syncwarp();
+}
+
 template <int EPI, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -225,21 +320,27 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const UmmaParams p)
 {
     constexpr bool GATEUP = (EPI == EPI_GATEUP);
-    constexpr int N_TILE = GATEUP ? 128 : BN;   // output columns per tile (gate and up share a tile)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
-    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES);
+    const uint32_t epi_bufs = tiles + STAGES * STAGE_BYTES;
+    SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES +
+                                               EPI_WARPS * EPI_BUF_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nk = p.status[ST_NK];
     const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
-    const int num_m = (M + BM - 1) / BM, num_n = (p.N + N_TILE - 1) / N_TILE;
+    const int num_m = (M + BM - 1) / BM;
+    // accumulator columns per tile; gate and up halves share a tile, so its output is half as wide
+    const int bn = GATEUP ? BN : choose_bn(num_m, p.N, gridDim.x, p.force_bn);
+    const int n_tile = GATEUP ? BN / 2 : bn;
+    const int num_n = (p.N + n_tile - 1) / n_tile;
     const int num_tiles = num_m * num_n;
     const int kb_per_seg = (K + BK - 1) / BK;
     const int num_kb = kb_per_seg * p.segments;
     const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
+    const int b_slabs = (bn + 63) / 64;    // 64-wide pieces of B loaded per stage
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -248,7 +349,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[s]), 4);
+            mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS);
         }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -271,10 +372,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             prefetch_tmap(&tmB);
             if (GATEUP || p.segments == 2) prefetch_tmap(&tmB2);
             if (p.segments == 2) prefetch_tmap(&tmA2);
+            const uint32_t stage_tx = A_BYTES + b_slabs * CHUNK_BYTES;
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * N_TILE;
+                const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * n_tile;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status,
                                    SITE_PRODUCER_EMPTY);
@@ -285,7 +387,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const CUtensorMap *mB = seg ? &tmB2 : &tmB;
                     const uint32_t bar = smem_u32(&ctl->full[stage]);
                     const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(bar, STAGE_BYTES);
+                    mbar_expect_tx(bar, stage_tx);
                     if (A_MN) {
 #pragma unroll
                         for (int j = 0; j < BM / 64; ++j)
@@ -293,15 +395,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     } else {
                         tma_load_2d(sa, mA, k0, m0, bar);
                     }
-                    if (B_MN) {
-#pragma unroll
-                        for (int j = 0; j < BN / 64; ++j)
+                    if (B_MN) {          // 64-column slabs of BK rows
+                        for (int j = 0; j < b_slabs; ++j)
                             tma_load_2d(sb + j * CHUNK_BYTES, mB, n0 + 64 * j, k0, bar);
-                    } else if (GATEUP) {
-                        tma_load_2d(sb, &tmB, k0, n0, bar);                 // 128 gate rows
-                        tma_load_2d(sb + B_BYTES / 2, &tmB2, k0, n0, bar);  // 128 up rows
-                    } else {
-                        tma_load_2d(sb, mB, k0, n0, bar);
+                    } else if (GATEUP) { // 128 gate rows, then 128 up rows, in 64-row pieces
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            tma_load_2d(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j, bar);
+                            tma_load_2d(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j, bar);
+                        }
+                    } else {             // 64-row pieces of a K-major tile are contiguous in smem
+                        for (int j = 0; j < b_slabs; ++j)
+                            tma_load_2d(sb + j * CHUNK_BYTES, mB, k0, n0 + 64 * j, bar);
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -310,7 +415,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && !zero_acc) {
-            constexpr uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0);
+            const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, bn);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
@@ -342,13 +447,39 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
-        const int quarter = warp & 3;                 // tensor-memory lanes 32*quarter .. +31
+        // Two warps share each 32-lane quarter of tensor memory and alternate over 32-column chunks.
+        const int ew = warp - 2;
+        const int quarter = warp & 3;
+        const int half = ew >> 2;
         const int row_in_tile = quarter * 32 + lane;
+        const uint32_t sbuf = epi_bufs + ew * EPI_BUF_BYTES;
+        const int esz = p.out_fp32 ? 4 : 2;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * N_TILE;
+            const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * n_tile;
             const int m = m0 + row_in_tile;
+            const int n_end = min(n0 + n_tile, p.N);
+            const bool row_valid = m < M;
+            int64_t tok = 0;
+            if ((EPI == EPI_DOWN || EPI == EPI_DX) && row_valid) tok = p.idx[m];
+            // prefetch of the per-row epilogue inputs of the first chunk (overlaps the accumulator wait)
+            uint4 pa[4], pb[4];
+            auto prefetch = [&](int n) {
+                if (EPI == EPI_DH || EPI == EPI_DOWN || EPI == EPI_DX) {
+                    const int64_t o = (int64_t)m * p.ldo + n;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        pa[v] = make_uint4(0, 0, 0, 0);
+                        pb[v] = make_uint4(0, 0, 0, 0);
+                        if (row_valid && n + v * 8 < n_end) {
+                            pa[v] = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o)[v];
+                            if (EPI == EPI_DH) pb[v] = reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o)[v];
+                        }
+                    }
+                }
+            };
+            prefetch(n0 + half * 32);
             if (!zero_acc) {
                 ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
                                SITE_EPI_TMEM_FULL);
@@ -356,123 +487,108 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 tc_fence_after();
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
-            const bool row_valid = m < M;
-            int64_t tok = 0;
-            if ((EPI == EPI_DOWN || EPI == EPI_DX) && row_valid) tok = p.idx[m];
 
 #pragma unroll 1
-            for (int c = 0; c < N_TILE / 32; ++c) {
-                const int n = n0 + c * 32;
-                uint32_t r[32], r2[32];
+            for (int n = n0 + half * 32; n < n_end; n += 64) {
+                const int col = n - n0;
+                uint32_t r[32], r2[GATEUP ? 32 : 1];
                 if (!zero_acc) {
-                    tmem_ld32(t_row + c * 32, r);
-                    if (GATEUP) tmem_ld32(t_row + 128 + c * 32, r2);
-                    tmem_ld_wait();
+                    tmem_ld32(t_row + col, r);
+                    if (GATEUP) tmem_ld32(t_row + BN / 2 + col, *reinterpret_cast<uint32_t(*)[32]>(&r2));
                 } else {
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) { r[q] = 0u; r2[q] = 0u; }
+                    for (int q = 0; q < 32; ++q) r[q] = 0u;
                 }
-                if (n >= p.N) continue;
-                const int64_t o = (int64_t)m * p.ldo + n;
+                uint4 ca[4], cb[4];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) { ca[v] = pa[v]; cb[v] = pb[v]; }
+                if (n + 64 < n_end) prefetch(n + 64);
+                if (!zero_acc) tmem_ld_wait();
+                const int valid_slots = min(4, (n_end - n) / 8);
+                uint32_t w[16];
                 if (EPI == EPI_GATEUP) {
                     // compacted G, U, H; rows past Nk inside the tile are written as zeros
-                    bf16 *G = (bf16 *)p.out0 + o, *U = (bf16 *)p.out1 + o, *H = (bf16 *)p.out2 + o;
+                    const int64_t o = (int64_t)m * p.ldo + n;
+                    char *rowG = (char *)((bf16 *)p.out0 + o), *rowU = (char *)((bf16 *)p.out1 + o),
+                         *rowH = (char *)((bf16 *)p.out2 + o);
+                    if (!row_valid) {
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        if (n + v * 8 >= p.N) break;
-                        uint32_t wg[4], wu[4], wh[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            float g0 = __uint_as_float(r[v * 8 + 2 * q]), g1 = __uint_as_float(r[v * 8 + 2 * q + 1]);
-                            float u0 = __uint_as_float(r2[v * 8 + 2 * q]), u1 = __uint_as_float(r2[v * 8 + 2 * q + 1]);
-                            if (!row_valid) { g0 = g1 = u0 = u1 = 0.0f; }
-                            wg[q] = pack_bf16(g0, g1);
-                            wu[q] = pack_bf16(u0, u1);
-                            wh[q] = pack_bf16(swiglu(g0, u0), swiglu(g1, u1));
-                        }
-                        reinterpret_cast<uint4 *>(G)[v] = make_uint4(wg[0], wg[1], wg[2], wg[3]);
-                        reinterpret_cast<uint4 *>(U)[v] = make_uint4(wu[0], wu[1], wu[2], wu[3]);
-                        reinterpret_cast<uint4 *>(H)[v] = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                        for (int q = 0; q < 32; ++q) { r[q] = 0u; r2[GATEUP ? q : 0] = 0u; }
                     }
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) w[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+                    store_rows_64B(sbuf, lane, w, rowG, valid_slots);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        w[q] = pack_bf16(__uint_as_float(r2[GATEUP ? 2 * q : 0]), __uint_as_float(r2[GATEUP ? 2 * q + 1 : 0]));
+                    store_rows_64B(sbuf, lane, w, rowU, valid_slots);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        w[q] = pack_bf16(fast_swiglu(__uint_as_float(r[2 * q]), __uint_as_float(r2[GATEUP ? 2 * q : 0])),
+                                         fast_swiglu(__uint_as_float(r[2 * q + 1]), __uint_as_float(r2[GATEUP ? 2 * q + 1 : 0])));
+                    store_rows_64B(sbuf, lane, w, rowH, valid_slots);
                 } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
                     // residual add in fp32, one rounding, scatter to the token's row
-                    if (row_valid) {
-                        const uint4 *res = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o);
-                        uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)p.out0 + tok * p.ldo + n);
+                    const uint32_t rw[16] = {ca[0].x, ca[0].y, ca[0].z, ca[0].w, ca[1].x, ca[1].y, ca[1].z, ca[1].w,
+                                             ca[2].x, ca[2].y, ca[2].z, ca[2].w, ca[3].x, ca[3].y, ca[3].z, ca[3].w};
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        float a0, a1;
+                        unpack_bf16(rw[q], a0, a1);
+                        w[q] = pack_bf16(a0 + __uint_as_float(r[2 * q]), a1 + __uint_as_float(r[2 * q + 1]));
+                    }
+                    char *row = row_valid ? (char *)((bf16 *)p.out0 + tok * p.ldo + n) : nullptr;
+                    store_rows_64B(sbuf, lane, w, row, valid_slots);
+                } else if (EPI == EPI_DH) {
+                    const uint32_t gw[16] = {ca[0].x, ca[0].y, ca[0].z, ca[0].w, ca[1].x, ca[1].y, ca[1].z, ca[1].w,
+                                             ca[2].x, ca[2].y, ca[2].z, ca[2].w, ca[3].x, ca[3].y, ca[3].z, ca[3].w};
+                    const uint32_t uw[16] = {cb[0].x, cb[0].y, cb[0].z, cb[0].w, cb[1].x, cb[1].y, cb[1].z, cb[1].w,
+                                             cb[2].x, cb[2].y, cb[2].z, cb[2].w, cb[3].x, cb[3].y, cb[3].z, cb[3].w};
+                    uint32_t w2[16];
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) {
+                        float g0, g1, u0, u1, dg0, dg1, du0, du1;
+                        unpack_bf16(gw[q], g0, g1);
+                        unpack_bf16(uw[q], u0, u1);
+                        fast_swiglu_bwd(__uint_as_float(r[2 * q]), g0, u0, dg0, du0);
+                        fast_swiglu_bwd(__uint_as_float(r[2 * q + 1]), g1, u1, dg1, du1);
+                        if (!row_valid) { dg0 = dg1 = du0 = du1 = 0.0f; }
+                        w[q] = pack_bf16(dg0, dg1);
+                        w2[q] = pack_bf16(du0, du1);
+                    }
+                    const int64_t o = (int64_t)m * p.ldo + n;
+                    store_rows_64B(sbuf, lane, w, (char *)((bf16 *)p.out0 + o), valid_slots);
+                    store_rows_64B(sbuf, lane, w2, (char *)((bf16 *)p.out1 + o), valid_slots);
+                } else {   // EPI_DW: weight-gradient tile, overwrite or accumulate
+                    const int64_t o = (int64_t)m * p.ldo + n;
+                    char *row = row_valid ? (char *)p.out0 + o * esz : nullptr;
+                    if (p.out_fp32) {
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) w[q] = r[hh * 16 + q];
+                            store_rows_64B_f32(sbuf, lane, w, row ? row + hh * 64 : nullptr,
+                                               min(4, max(0, (n_end - n - hh * 16) / 4)), p.accumulate);
+                        }
+                    } else if (!p.accumulate) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) w[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+                        store_rows_64B(sbuf, lane, w, row, valid_slots);
+                    } else if (row_valid) {   // bf16 accumulation: add in fp32, round once (per-row path)
+                        uint4 *dst = reinterpret_cast<uint4 *>(row);
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
-                            if (n + v * 8 >= p.N) break;
-                            uint4 rv = res[v];
-                            uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w}, ow[4];
+                            if (v >= valid_slots) break;
+                            uint4 old = dst[v];
+                            uint32_t oldw[4] = {old.x, old.y, old.z, old.w}, ow[4];
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 float a0, a1;
-                                unpack_bf16(rw[q], a0, a1);
+                                unpack_bf16(oldw[q], a0, a1);
                                 ow[q] = pack_bf16(a0 + __uint_as_float(r[v * 8 + 2 * q]),
                                                   a1 + __uint_as_float(r[v * 8 + 2 * q + 1]));
                             }
                             dst[v] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-                        }
-                    }
-                } else if (EPI == EPI_DH) {
-                    const uint4 *Gp = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o);
-                    const uint4 *Up = reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o);
-                    uint4 *dG = reinterpret_cast<uint4 *>((bf16 *)p.out0 + o);
-                    uint4 *dU = reinterpret_cast<uint4 *>((bf16 *)p.out1 + o);
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        if (n + v * 8 >= p.N) break;
-                        uint4 gv = make_uint4(0, 0, 0, 0), uv = gv;
-                        if (row_valid) { gv = Gp[v]; uv = Up[v]; }
-                        uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
-                        uint32_t og[4], ou[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            float g0, g1, u0, u1, dg0, dg1, du0, du1;
-                            unpack_bf16(gw[q], g0, g1);
-                            unpack_bf16(uw[q], u0, u1);
-                            swiglu_bwd(__uint_as_float(r[v * 8 + 2 * q]), g0, u0, dg0, du0);
-                            swiglu_bwd(__uint_as_float(r[v * 8 + 2 * q + 1]), g1, u1, dg1, du1);
-                            if (!row_valid) { dg0 = dg1 = du0 = du1 = 0.0f; }
-                            og[q] = pack_bf16(dg0, dg1);
-                            ou[q] = pack_bf16(du0, du1);
-                        }
-                        dG[v] = make_uint4(og[0], og[1], og[2], og[3]);
-                        dU[v] = make_uint4(ou[0], ou[1], ou[2], ou[3]);
-                    }
-                } else {   // EPI_DW: weight-gradient tile, overwrite or accumulate
-                    if (row_valid) {
-                        if (p.out_fp32) {
-                            float4 *dst = reinterpret_cast<float4 *>((float *)p.out0 + o);
-#pragma unroll
-                            for (int v = 0; v < 8; ++v) {
-                                if (n + v * 4 >= p.N) break;
-                                float4 w = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                       __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
-                                if (p.accumulate) {
-                                    float4 old = dst[v];
-                                    w.x += old.x; w.y += old.y; w.z += old.z; w.w += old.w;
-                                }
-                                dst[v] = w;
-                            }
-                        } else {
-                            uint4 *dst = reinterpret_cast<uint4 *>((bf16 *)p.out0 + o);
-#pragma unroll
-                            for (int v = 0; v < 4; ++v) {
-                                if (n + v * 8 >= p.N) break;
-                                uint32_t ow[4];
-                                uint4 old = make_uint4(0, 0, 0, 0);
-                                if (p.accumulate) old = dst[v];
-                                uint32_t oldw[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    float a0, a1;
-                                    unpack_bf16(oldw[q], a0, a1);
-                                    ow[q] = pack_bf16(a0 + __uint_as_float(r[v * 8 + 2 * q]),
-                                                      a1 + __uint_as_float(r[v * 8 + 2 * q + 1]));
-                                }
-                                dst[v] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
-                            }
                         }
                     }
                 }
@@ -570,22 +686,27 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
         return make_map(m, base, (int64_t)g.K, outer_rows, ld_mn, box_rows_kmajor);
     };
     ok &= mk(&mA, g.A, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM);
-    ok &= mk(&mB, g.B, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, gateup ? 128 : BN);
+    ok &= mk(&mB, g.B, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, 64);
     if (g.A2) ok &= mk(&mA2, g.A2, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM); else mA2 = mA;
-    if (g.B2) ok &= mk(&mB2, g.B2, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, gateup ? 128 : BN); else mB2 = mB;
+    if (g.B2) ok &= mk(&mB2, g.B2, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, 64); else mB2 = mB;
     if (!ok) return cudaErrorInvalidValue;
 
     UmmaParams p;
     p.M = g.M; p.N = g.N; p.K = g.K;
     p.m_from_nk = g.m_from_nk; p.k_from_nk = g.k_from_nk;
     p.segments = epi == EPI_DX ? 2 : 1;
+    p.force_bn = 0;
+    if (const char *e = getenv("SKIPFFN_TILE_N")) {   // tuning override: accumulator columns per tile
+        int v = atoi(e);
+        if (v >= 16 && v <= BN && v % 16 == 0) p.force_bn = v;
+    }
     p.status = const_cast<int32_t *>(g.status);
     p.idx = g.idx;
     p.out0 = g.out0; p.out1 = g.out1; p.out2 = g.out2;
     p.in0 = g.in0; p.in1 = g.in1;
     p.ldo = g.ldo; p.accumulate = g.accumulate; p.out_fp32 = g.out_fp32;
 
-    const int n_tile = gateup ? 128 : BN;
+    const int n_tile = 128;   // narrowest tile the kernel may choose
     const int64_t max_tiles = ((int64_t)g.M + BM - 1) / BM * (((int64_t)g.N + n_tile - 1) / n_tile);
     int grid = (int)(max_tiles < g_num_sms ? max_tiles : g_num_sms);
     if (grid <= 0) return cudaSuccess;

@@ -95,6 +95,14 @@ def test_multi_tile_ragged(dtype, path):
     _compare(w, run(w, path=path), _oracle_all(w))
 
 
+@pytest.mark.parametrize("tile_n", [128, 144, 176, 192, 240, 256])
+def test_every_tile_width(tile_n, monkeypatch):
+    # the device picks the accumulator width per launch; force each candidate class in turn
+    monkeypatch.setenv("SKIPFFN_TILE_N", str(tile_n))
+    w = wl.small_case(21, "bf16", 576, 1000, 3, 20, 200, 0.6)
+    _compare(w, run(w), _oracle_all(w))
+
+
 def test_contiguous_span_layout():
     # the paper's layout: one contiguous skipped span per sequence
     w = wl.uniform_batch(2, "bf16", 256, 512, 4, 10, 150, 10, skip_ratio=0.8, contiguous_span=True)
