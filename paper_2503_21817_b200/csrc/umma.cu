@@ -2,18 +2,26 @@
 // tcgen05.mma with fp32 accumulators in tensor memory, fused Skip-FFN epilogues.
 //
 // One persistent kernel template serves every contraction of the path:
-//   C[m, n] = sum_k A(m, k) * B(n, k),   tile 128 (M) x 256 (N) x 64 (K), bf16 in, fp32 accumulate.
+//   C[m, n] = sum_k A(m, k) * B(n, k),   bf16 in, fp32 accumulate, K step 64.
 // Either operand may be K-major (global array [rows = M or N, cols = K]) or MN-major (global array
 // [rows = K, cols = M or N]); the latter is what the backward pass needs for W_down (dH), for
 // W_gate / W_up (dX) and for both operands of the weight-gradient GEMMs, whose reduction axis is the
 // compacted token axis.
 //
-// Warp roles (192 threads, one CTA per SM):
-//   warp 0      TMA producer: fills a 4-stage ring of {A 128x64, B 256x64} tiles (128-byte swizzle)
-//   warp 1      MMA issuer: owns the tensor-memory allocation (512 columns = two 128x256 fp32
-//               accumulators), issues four K=16 tcgen05.mma per stage, releases stages and
-//               publishes finished accumulators through tcgen05.commit
-//   warps 2..5  epilogue: read one accumulator (tcgen05.ld, one row per thread) while the MMA warp
+// Two launch shapes share the code:
+//   PAIR   two CTAs of a cluster (an SM pair) compute one 256 x bn tile with cta_group::2 MMAs.
+//          Each CTA stages its own 128 rows of A and HALF of the B tile, so an SM pulls 32 KiB
+//          from L2 per K step for a 128 x 256 x 64 block of work (128 flop/byte); six stages.
+//   SINGLE one CTA computes a 128 x bn tile (48 KiB per K step, 85 flop/byte); four stages.
+//          Used when the device cannot co-schedule pairs.
+//
+// Warp roles (320 threads per CTA, one CTA per SM):
+//   warp 0      TMA producer: fills the stage ring (128-byte swizzle)
+//   warp 1      MMA issuer (the pair's leader CTA issues for both SMs): owns the tensor-memory
+//               allocation (512 columns = two 128 x 256 fp32 accumulators per SM), issues four K=16
+//               tcgen05.mma per stage, releases stages and publishes finished accumulators through
+//               tcgen05.commit
+//   warps 2..9  epilogue: read one accumulator (tcgen05.ld, one row per thread) while the MMA warp
 //               fills the other, apply the fused epilogue, write global memory
 //
 // The kept-token count Nk lives in device memory, so tile counts are derived on the device and no
@@ -27,18 +35,21 @@
 namespace skipffn {
 
 constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;             // 16 KiB
-constexpr int B_BYTES = BN * BK * 2;             // 32 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;   // 48 KiB
-constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64-wide MN-major slab of BK rows: 8 KiB
+constexpr int MAX_STAGES = 6;
+constexpr int A_BYTES = BM * BK * 2;             // 16 KiB: this CTA's 128 rows of A
+constexpr int CHUNK_BYTES = 64 * BK * 2;         // one 64-wide slab of B (or MN-major A): 8 KiB
 constexpr int ACC_COLS = 256;                    // fp32 columns per accumulator
 constexpr int TMEM_COLS = 512;
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 2048;              // per-warp staging: 32 rows x 64 B
 constexpr int UMMA_THREADS = 64 + 32 * EPI_WARPS;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES + 1024 /*alignment slack*/ +
-                           256 /*barriers*/;
+template <bool PAIR> struct Shape {
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr int B_BYTES = PAIR ? 128 * BK * 2 : 256 * BK * 2;   // B rows staged per CTA
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES +
+                                      1024 /*alignment slack*/ + 256 /*barriers*/;
+};
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s
 
 // ------------------------------------------------------------------------------------ PTX
@@ -169,6 +180,74 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- cluster (SM pair) variants
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on the pair leader's mbarrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1,
+                                                 uint32_t leader_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst),
+                 "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+                 : "memory");
+}
+// one MMA spanning both SMs of the pair: 256 rows (128 per SM), issued by the leader CTA
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                               uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on the mbarrier at this offset in BOTH CTAs of the pair once the MMAs issued so far retire
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"((uint16_t)3)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle (layout code 2), descriptor version 1.
 // K-major tile:  rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride byte offset).
 // MN-major tile: 64-wide slabs of BK rows x 128 B; 8-row groups 1024 B apart (stride byte offset),
@@ -184,11 +263,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n (a multiple of 16, at most 256).
-__host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major, int n)
+// Instruction descriptor: bf16 x bf16 -> fp32, M = m (128, or 256 across an SM pair), N = n (a
+// multiple of 16, at most 256).
+__host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major, int m, int n)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) |
-           ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------ kernel
@@ -197,6 +277,7 @@ struct UmmaParams {
     int32_t m_from_nk, k_from_nk;    // extent is the device-resident kept count
     int32_t segments;                // 2: second K segment reads tmA2 / tmB2 (dX)
     int32_t force_bn;                // > 0: tile width override (tuning)
+    int32_t force_stages;            // > 0: use fewer ring stages (tuning)
     int32_t *status;
     const int32_t *idx;
     void *out0, *out1, *out2;
@@ -206,7 +287,7 @@ struct UmmaParams {
 };
 
 struct alignas(8) SmemCtl {
-    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -237,16 +318,18 @@ __device__ __forceinline__ void fast_swiglu_bwd(float dh, float g, float u, floa
 // Tile width (accumulator columns) for this launch.  With few M tiles the tile count rarely fills
 // a whole number of waves of the persistent grid; narrower tiles trade MMA width for fewer idle
 // SMs in the last wave.  Cost model: waves x (MMA columns + B columns loaded, in 64-wide slabs).
-__device__ __forceinline__ int choose_bn(int num_m, int N, int grid, int force_bn)
+// `grid` = number of tile workers (CTAs, or CTA pairs); `split` = CTAs sharing the B tile.
+__device__ __forceinline__ int choose_bn(int num_m, int N, int grid, int force_bn, int split)
 {
     if (force_bn > 0) return force_bn;
+    if (force_bn == 0) return BN;
     int best = BN;
     long best_cost = -1;
-    for (int bn = BN; bn >= 128; bn -= 16) {
+    for (int bn = BN; bn >= 128; bn -= 16 * split) {
         const int num_n = (N + bn - 1) / bn;
         const long tiles = (long)num_m * num_n;
         const long waves = (tiles + grid - 1) / grid;
-        const long cost = waves * (bn + 64 * ((bn + 63) / 64) + 32);
+        const long cost = waves * (bn + 64 * split * ((bn / split + 63) / 64) + 32);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
     }
     return best;
@@ -313,13 +396,17 @@ __device__ __forceinline__ void store_rows_64B_f32(uint32_t sbuf, int lane, cons
     __syncwarp();
 }
 
-template <int EPI, bool A_MN, bool B_MN>
+template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
             const UmmaParams p)
 {
     constexpr bool GATEUP = (EPI == EPI_GATEUP);
+    constexpr int STAGES = Shape<PAIR>::STAGES;
+    constexpr int STAGE_BYTES = Shape<PAIR>::STAGE_BYTES;
+    constexpr int SPLIT = PAIR ? 2 : 1;           // CTAs sharing one tile
+    constexpr int TILE_M = BM * SPLIT;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -328,19 +415,24 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                                EPI_WARPS * EPI_BUF_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // position in the SM pair; 0 leads
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int num_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int nk = p.status[ST_NK];
     const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
-    const int num_m = (M + BM - 1) / BM;
+    const int num_m = (M + TILE_M - 1) / TILE_M;
     // accumulator columns per tile; gate and up halves share a tile, so its output is half as wide
-    const int bn = GATEUP ? BN : choose_bn(num_m, p.N, gridDim.x, p.force_bn);
+    const int bn = GATEUP ? BN : choose_bn(num_m, p.N, num_workers, p.force_bn, SPLIT);
     const int n_tile = GATEUP ? BN / 2 : bn;
     const int num_n = (p.N + n_tile - 1) / n_tile;
     const int num_tiles = num_m * num_n;
     const int kb_per_seg = (K + BK - 1) / BK;
     const int num_kb = kb_per_seg * p.segments;
     const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
-    const int b_slabs = (bn + 63) / 64;    // 64-wide pieces of B loaded per stage
+    const int bn_cta = bn / SPLIT;         // B rows (tile columns) this CTA stages
+    const int b_slabs = (bn_cta + 63) / 64;
+    const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -349,18 +441,19 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS);
+            mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS * SPLIT);
         }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
-        tmem_relinquish();
+        if (PAIR) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish_pair(); }
+        else      { tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish(); }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     volatile int *abort_flag = &ctl->abort_flag;
@@ -372,11 +465,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             prefetch_tmap(&tmB);
             if (GATEUP || p.segments == 2) prefetch_tmap(&tmB2);
             if (p.segments == 2) prefetch_tmap(&tmA2);
-            const uint32_t stage_tx = A_BYTES + b_slabs * CHUNK_BYTES;
+            // bytes landing on the (leader's) full barrier per stage, from every CTA of the tile
+            const uint32_t stage_tx = SPLIT * (A_BYTES + b_slabs * CHUNK_BYTES);
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * n_tile;
+            for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
+                const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
+                const int n0 = (tile / num_m) * n_tile;
+                const int nb0 = GATEUP ? n0 : n0 + (int)rank * bn_cta;   // first B row of this CTA
                 for (int kb = 0; kb < num_kb; ++kb) {
                     ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status,
                                    SITE_PRODUCER_EMPTY);
@@ -385,40 +481,46 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     const int k0 = (kb - seg * kb_per_seg) * BK;
                     const CUtensorMap *mA = seg ? &tmA2 : &tmA;
                     const CUtensorMap *mB = seg ? &tmB2 : &tmB;
-                    const uint32_t bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t own_bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
                     const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    mbar_expect_tx(bar, stage_tx);
+                    auto load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1) {
+                        if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar);
+                        else tma_load_2d(dst, map, c0, c1, bar);
+                    };
+                    if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
                     if (A_MN) {
 #pragma unroll
-                        for (int j = 0; j < BM / 64; ++j)
-                            tma_load_2d(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0, bar);
+                        for (int j = 0; j < BM / 64; ++j) load(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0);
                     } else {
-                        tma_load_2d(sa, mA, k0, m0, bar);
+                        load(sa, mA, k0, m0);
                     }
                     if (B_MN) {          // 64-column slabs of BK rows
-                        for (int j = 0; j < b_slabs; ++j)
-                            tma_load_2d(sb + j * CHUNK_BYTES, mB, n0 + 64 * j, k0, bar);
+                        for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, nb0 + 64 * j, k0);
+                    } else if (GATEUP && PAIR) {   // leader stages the 128 gate rows, its peer the up rows
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)
+                            load(sb + j * CHUNK_BYTES, rank == 0 ? &tmB : &tmB2, k0, n0 + 64 * j);
                     } else if (GATEUP) { // 128 gate rows, then 128 up rows, in 64-row pieces
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            tma_load_2d(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j, bar);
-                            tma_load_2d(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j, bar);
+                            load(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j);
+                            load(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j);
                         }
                     } else {             // 64-row pieces of a K-major tile are contiguous in smem
-                        for (int j = 0; j < b_slabs; ++j)
-                            tma_load_2d(sb + j * CHUNK_BYTES, mB, k0, n0 + 64 * j, bar);
+                        for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
                     }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    if (++stage == nst) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && !zero_acc) {
-            const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, bn);
+        if (lane == 0 && !zero_acc && rank == 0) {
+            const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, TILE_M, bn);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
                 ok = mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1, abort_flag, p.status,
                                SITE_MMA_TMEM_EMPTY);
                 if (!ok) break;
@@ -436,12 +538,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                                  : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
                         const uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
                                                  : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-                        umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
+                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0);
+                        else umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
                     }
-                    umma_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs retire
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                    // the stage is reusable (in both CTAs) once these MMAs retire
+                    if (PAIR) umma_commit_pair(smem_u32(&ctl->empty[stage]));
+                    else umma_commit(smem_u32(&ctl->empty[stage]));
+                    if (++stage == nst) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit(smem_u32(&ctl->tmem_full[acc]));
+                if (ok) {
+                    if (PAIR) umma_commit_pair(smem_u32(&ctl->tmem_full[acc]));
+                    else umma_commit(smem_u32(&ctl->tmem_full[acc]));
+                }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
         }
@@ -456,8 +564,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int esz = p.out_fp32 ? 4 : 2;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-            const int m0 = (tile % num_m) * BM, n0 = (tile / num_m) * n_tile;
+        // accumulators are handed back on the leader's barrier, which its MMA warp waits on
+        const uint32_t empty_bar0 = smem_u32(&ctl->tmem_empty[0]);
+        for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
+            const int m0 = (tile % num_m) * TILE_M + (int)rank * BM, n0 = (tile / num_m) * n_tile;
             const int m = m0 + row_in_tile;
             const int n_end = min(n0 + n_tile, p.N);
             const bool row_valid = m < M;
@@ -596,7 +706,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (!zero_acc) {
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+                if (lane == 0) {
+                    const uint32_t bar = empty_bar0 + acc * 8;
+                    if (PAIR) mbar_arrive_cluster(mapa_rank(bar, 0));
+                    else mbar_arrive(bar);
+                }
             }
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
@@ -605,9 +719,11 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ---------------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // neither SM leaves while the other may still touch its memory
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+        else tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -649,19 +765,63 @@ static bool make_map(CUtensorMap *m, const void *base, int64_t inner, int64_t ou
 
 static int g_num_sms = 0;
 
-template <int EPI, bool A_MN, bool B_MN>
+// Launch one instantiation.  PAIR kernels run as clusters of two CTAs; `workers` counts tiles
+// processed concurrently (CTAs, or CTA pairs).
+template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
-                            const CUtensorMap &b2, const UmmaParams &p, int grid, cudaStream_t s)
+                            const CUtensorMap &b2, const UmmaParams &p, int64_t max_tiles,
+                            cudaStream_t s)
 {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(k_umma_gemm<EPI, A_MN, B_MN>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    constexpr int SMEM = Shape<PAIR>::SMEM_BYTES;
+    static int max_workers = -1;   // -1 not yet queried; 0 unavailable
+    auto kern = k_umma_gemm<EPI, A_MN, B_MN, PAIR>;
+    if (max_workers < 0) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        if (PAIR) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3(2 * g_num_sms);
+            q.blockDim = dim3(UMMA_THREADS);
+            q.dynamicSmemBytes = SMEM;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            q.attrs = at; q.numAttrs = 1;
+            int n = 0;
+            e = cudaOccupancyMaxActiveClusters(&n, kern, &q);
+            if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+            max_workers = n;
+        } else {
+            max_workers = g_num_sms;
+        }
     }
-    k_umma_gemm<EPI, A_MN, B_MN><<<grid, UMMA_THREADS, SMEM_BYTES, s>>>(a, b, a2, b2, p);
-    return cudaGetLastError();
+    if (max_workers <= 0) return cudaErrorNotSupported;
+    const int workers = (int)(max_tiles < max_workers ? max_tiles : max_workers);
+    if (workers <= 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
+    cfg.blockDim = dim3(UMMA_THREADS);
+    cfg.dynamicSmemBytes = SMEM;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = PAIR ? 2 : 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, a, b, a2, b2, p);
+}
+
+template <bool PAIR>
+static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
+                            const CUtensorMap &b2, const UmmaParams &p, int64_t max_tiles, cudaStream_t s)
+{
+    switch (epi) {
+    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    case EPI_DH:     return launch_k<EPI_DH, false, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    case EPI_DX:     return launch_k<EPI_DX, false, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    default: return cudaErrorInvalidValue;
+    }
 }
 
 // GemmArgs conventions: an operand with ld_k == 1 is K-major ([outer = M or N rows, inner = K]),
@@ -696,9 +856,11 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
     p.m_from_nk = g.m_from_nk; p.k_from_nk = g.k_from_nk;
     p.segments = epi == EPI_DX ? 2 : 1;
     p.force_bn = 0;
+    p.force_stages = 0;
+    if (const char *e = getenv("SKIPFFN_STAGES")) p.force_stages = atoi(e);
     if (const char *e = getenv("SKIPFFN_TILE_N")) {   // tuning override: accumulator columns per tile
         int v = atoi(e);
-        if (v >= 16 && v <= BN && v % 16 == 0) p.force_bn = v;
+        if (v >= 32 && v <= BN && v % 32 == 0) p.force_bn = v;
     }
     p.status = const_cast<int32_t *>(g.status);
     p.idx = g.idx;
@@ -706,19 +868,19 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
     p.in0 = g.in0; p.in1 = g.in1;
     p.ldo = g.ldo; p.accumulate = g.accumulate; p.out_fp32 = g.out_fp32;
 
+    // SM pairs by default; SKIPFFN_SINGLE_CTA=1 (or a device that cannot co-schedule pairs) selects
+    // the one-CTA-per-tile shape
+    static int single = -1;
+    if (single < 0) { const char *e = getenv("SKIPFFN_SINGLE_CTA"); single = (e && atoi(e) != 0) ? 1 : 0; }
     const int n_tile = 128;   // narrowest tile the kernel may choose
-    const int64_t max_tiles = ((int64_t)g.M + BM - 1) / BM * (((int64_t)g.N + n_tile - 1) / n_tile);
-    int grid = (int)(max_tiles < g_num_sms ? max_tiles : g_num_sms);
-    if (grid <= 0) return cudaSuccess;
-
-    switch (epi) {
-    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false>(mA, mB, mA2, mB2, p, grid, s);
-    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false>(mA, mB, mA2, mB2, p, grid, s);
-    case EPI_DH:     return launch_k<EPI_DH, false, true>(mA, mB, mA2, mB2, p, grid, s);
-    case EPI_DW:     return launch_k<EPI_DW, true, true>(mA, mB, mA2, mB2, p, grid, s);
-    case EPI_DX:     return launch_k<EPI_DX, false, true>(mA, mB, mA2, mB2, p, grid, s);
-    default: return cudaErrorInvalidValue;
+    const int64_t n_tiles = ((int64_t)g.N + n_tile - 1) / n_tile;
+    if (!single) {
+        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + 2 * BM - 1) / (2 * BM) * n_tiles, s);
+        if (e != cudaErrorNotSupported) return e;
+        (void)cudaGetLastError();
+        single = 1;
     }
+    return dispatch<false>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + BM - 1) / BM * n_tiles, s);
 }
 
 }  // namespace skipffn
