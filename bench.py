@@ -165,6 +165,36 @@ def workload_config(args, w):
             "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
 
 
+# ------------------------------------------------------------------------------ rank aggregation
+def max_over_ranks(ms, device=None):
+    """Slowest rank's time: replicas finish when the last one does."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(units, device=None):
+    """Units (kept tokens) processed per step by the whole job."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return int(units)
+    t = torch.tensor([units], device=device, dtype=torch.int64)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return int(t.item())
+
+
+def job_throughput(units_local, ms_local, steps, device=None):
+    """(kept tokens/s of the whole job, ms per step): all ranks' units over the slowest rank's time."""
+    ms = max_over_ranks(ms_local, device)
+    units = sum_over_ranks(units_local, device)
+    return units / (ms / steps * 1e-3), ms / steps
+
+
 # ------------------------------------------------------------------------------ our arm
 def run_ours(args):
     import torch
@@ -225,12 +255,7 @@ def run_ours(args):
         e1.record()
         barrier()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, t0, t1
+        return e0.elapsed_time(e1), t0, t1
 
     if args.profile_only:      # short launch sequence for ncu: W + K steps, nothing else
         for _ in range(args.warmup + args.steps):
@@ -255,16 +280,16 @@ def run_ours(args):
     prof = ctx.profile(step, args.steps) if hasattr(ctx, "profile") else None
     ctx.poll()
 
+    # whole-job numbers: every rank's kept tokens over the slowest rank's time
+    value, ms_step = job_throughput(nk, ms, args.steps, dev)
+    value_e2e, ms_step_e2e = job_throughput(nk, ms_e2e, args.steps, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     pk = peaks()
-    ms_step = ms / args.steps
-    flops = sk.skipffn_flops(C, I, nk)
-    value = world * nk / (ms_step * 1e-3)
-    tflops = world * flops / (ms_step * 1e-3) / 1e12
+    tflops = value * sk.skipffn_flops(C, I, 1) / 1e12
     unit_flops = 2.0 * nk * C * I     # one GEMM "unit" of the path: 2 * Nk * C * I
     kernel_units = {"gateup": 2, "down": 1, "dh": 1, "dw_down": 1, "dw_gate": 1, "dw_up": 1, "dx": 2}
     kernels, roofline = {}, None
@@ -302,8 +327,8 @@ def run_ours(args):
             "frac_of_measured_bf16_peak": tflops / world / pk["bf16_tflops"],
             "frac_of_sustained_bf16_peak": (tflops / world / pk["bf16_tflops_sustained"]) if pk["bf16_tflops_sustained"] else None,
             "frac_of_nominal_bf16_peak": tflops / world / 2250.0,
-            "e2e": {"value": world * nk / (ms_e2e / args.steps * 1e-3), "unit": UNIT,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+            "e2e": {"value": value_e2e, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_step_e2e},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
             "kernels": kernels, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
