@@ -132,6 +132,33 @@ double skipffn_flops(const skipffn_config *cfg, int64_t n_kept);
 
 const char *skipffn_strerror(skipffn_status status);
 
+/* Kept-row index list without a workspace or a handle, for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: it is a packaging of the mask compaction above, useful
+ * by itself e.g. to drop the skipped tokens' rows from a key/value cache.)
+ *
+ * Who needs it: code running where cudaMalloc is not an option -- a process whose framework has
+ * already reserved all device memory for its own pool, a latency-critical loop that cannot take
+ * cudaMalloc's device-wide synchronisation, or a host application that forbids allocation calls
+ * from extensions.  The kernel's scratch (token -> rank map and kept count) lives in a fixed
+ * array inside the library image, about 256 KiB per device that loads the library, held until
+ * the process exits.  The call allocates nothing, on the device or through any library.
+ *
+ * skip_mask : [N] bytes on the device, nonzero = skipped.
+ * idx       : [N] int32 on the device; entries 0 .. Nk-1 receive the ascending indices of the kept
+ *             tokens, the remaining entries are unspecified.
+ * nk        : one int32 on the device, receives Nk.
+ * Work is enqueued on `stream`; nothing is synchronised.
+ *
+ * N > SKIPFFN_STATIC_MAX_TOKENS returns SKIPFFN_EUNSUPPORTED and launches nothing.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.
+ * All calls on a device share the array: calls that may overlap on the GPU (different streams or
+ * host threads) race and must be serialised by the caller.  Nothing in it has to be zero between
+ * calls; each call overwrites every word it reads. */
+#define SKIPFFN_STATIC_MAX_TOKENS 65536
+skipffn_status skipffn_compact_static(const uint8_t *skip_mask, int64_t N, int32_t *idx,
+                                      int32_t *nk, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

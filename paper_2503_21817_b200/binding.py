@@ -16,7 +16,9 @@ _lib: Optional[ctypes.CDLL] = None
 EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_destroy",
            "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
-           "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read"]
+           "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
+           "skipffn_compact_static"]
+STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
                  "dw_up", "dx"]
@@ -72,6 +74,8 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_profile_enable.argtypes = [vp, i32]
     lib.skipffn_profile_read.restype = i32
     lib.skipffn_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.skipffn_compact_static.restype = i32
+    lib.skipffn_compact_static.argtypes = [vp, i64, vp, vp, vp]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -99,6 +103,31 @@ def skipffn_strerror(status: int) -> str:
 
 def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def skipffn_compact_static(skip_mask, idx, nk) -> None:
+    """Kept-row list for callers that cannot allocate device memory (``skipffn_compact_static``).
+
+    All three arguments are CUDA tensors the caller already owns: ``skip_mask`` uint8 ``[N]``,
+    ``idx`` int32 with at least N entries (the first Nk receive the ascending kept indices), ``nk``
+    int32 with one entry.  Neither this wrapper nor the library call allocates anything; the
+    kernel's scratch is a fixed array inside the library, which limits N to ``STATIC_MAX_TOKENS``
+    and means that calls overlapping on the GPU must be serialised by the caller.  Enqueued on the
+    current torch stream."""
+    import torch
+    N = skip_mask.numel()
+    if skip_mask.dtype != torch.uint8 or idx.dtype != torch.int32 or nk.dtype != torch.int32:
+        raise ValueError("skip_mask must be uint8, idx and nk int32")
+    if not (skip_mask.is_cuda and idx.is_cuda and nk.is_cuda and skip_mask.is_contiguous()
+            and idx.is_contiguous()) or idx.numel() < N or nk.numel() < 1:
+        raise ValueError("skip_mask, idx (>= N entries) and nk (1 entry) must be contiguous CUDA tensors")
+    stream = ctypes.c_void_p(torch.cuda.current_stream(skip_mask.device).cuda_stream)
+    st = load_library().skipffn_compact_static(_ptr(skip_mask), N, _ptr(idx), _ptr(nk), stream)
+    if st == 2:
+        raise SkipFFNError(st, f"skipffn_compact_static: N = {N} exceeds the fixed scratch of "
+                               f"{STATIC_MAX_TOKENS} tokens")
+    if st != 0:
+        raise SkipFFNError(st, "skipffn_compact_static")
 
 
 class SkipFFN:
