@@ -38,7 +38,21 @@ KERNEL_NAMES = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_
                 "dw_up", "dx"]
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each GEMM kernel at the
 # default workload, from the ncu captures summarised under profiles/; None until captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"gateup": 368.7e6, "down": 235.7e6, "dh": 301.9e6, "dw_down": 129.0e6,
+                     "dw_gate": 170.3e6, "dw_up": 170.1e6, "dx": 451.0e6}
+# sha256 prefix of csrc/umma.cu when those counters were taken; once the kernel source differs the
+# counters no longer describe it and `traffic` is reported as null
+NCU_TRAFFIC_SOURCE_SHA = "faef05494660a744"
+
+
+def ncu_traffic(kernel):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2503_21817_b200", "csrc", "umma.cu")
+    try:
+        cur = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return NCU_TRAFFIC_BYTES.get(kernel) if cur == NCU_TRAFFIC_SOURCE_SHA else None
 
 
 def peaks():
@@ -306,7 +320,7 @@ def run_ours(args):
         roofline = {"kernel": f"k_umma_gemm[{top}]", "bound": "tensor", "achieved": gemms[top]["tflops"],
                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemms[top]["tflops"] / pk["bf16_tflops"],
                     "peak_source": pk["source"] + " (burst cuBLAS bf16)",
-                    "traffic": NCU_TRAFFIC_BYTES.get(top),
+                    "traffic": ncu_traffic(top),
                     "all_gemm_kernels": {"tflops": sum(kernel_units.values()) * unit_flops /
                                          (sum(v["ms"] for v in gemms.values()) * 1e-3) / 1e12}}
         roofline["all_gemm_kernels"]["frac"] = roofline["all_gemm_kernels"]["tflops"] / pk["bf16_tflops"]
