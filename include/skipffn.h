@@ -126,6 +126,17 @@ skipffn_status skipffn_profile_read(skipffn_saved *saved, float *ms);
 /* Number of kernels the last forward (which=0) or backward (which=1) call enqueued. */
 int32_t skipffn_last_launches(const skipffn_saved *saved, int32_t which);
 
+/* Diagnostic (host only, launches nothing): the work distribution of the tensor-core GEMM kernels.
+ * A launch with `tiles` output tiles of `k_blocks` K-blocks each runs on `workers` persistent
+ * workers; whole waves of tiles are handed out tile by tile, the tiles of the last one-to-two waves
+ * are cut along K into equal runs (split_k != 0).  Returns the number of segments of `worker`'s
+ * schedule (-1 on bad arguments) and, for 0 <= i < that number, writes segment i to seg[5] =
+ * {tile, first K-block, end K-block, partial, first source worker}: partial = 1 means the run stops
+ * before the tile's last K-block and its accumulator is handed over; otherwise the worker finishes
+ * the tile after adding the accumulators handed over by workers seg[4] .. worker-1. */
+int32_t skipffn_schedule_segment(int32_t workers, int32_t tiles, int32_t k_blocks, int32_t split_k,
+                                 int32_t worker, int32_t i, int32_t *seg);
+
 /* Algorithmic floating-point operations of one forward+backward call with n_kept kept tokens:
  * 18 * n_kept * C * I (forward 6: three GEMMs of the section 6.2 cost model; backward 12). */
 double skipffn_flops(const skipffn_config *cfg, int64_t n_kept);

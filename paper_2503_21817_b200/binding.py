@@ -17,7 +17,7 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
            "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
-           "skipffn_compact_static"]
+           "skipffn_compact_static", "skipffn_schedule_segment"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.skipffn_compact_static.restype = i32
     lib.skipffn_compact_static.argtypes = [vp, i64, vp, vp, vp]
+    lib.skipffn_schedule_segment.restype = i32
+    lib.skipffn_schedule_segment.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -99,6 +101,21 @@ def skipffn_flops(C, I, n_kept) -> float:
 
 def skipffn_strerror(status: int) -> str:
     return load_library().skipffn_strerror(int(status)).decode()
+
+
+def skipffn_schedule(workers: int, tiles: int, k_blocks: int, split_k: bool, worker: int):
+    """Segments ``(tile, kb0, kb1, partial, src_lo)`` of one worker's schedule, in processing order
+    (``skipffn_schedule_segment``; host only)."""
+    lib = load_library()
+    seg = (ctypes.c_int32 * 5)()
+    n = lib.skipffn_schedule_segment(workers, tiles, k_blocks, int(split_k), worker, -1, seg)
+    if n < 0:
+        raise SkipFFNError(1, "skipffn_schedule_segment")
+    out = []
+    for i in range(n):
+        lib.skipffn_schedule_segment(workers, tiles, k_blocks, int(split_k), worker, i, seg)
+        out.append(tuple(seg))
+    return out
 
 
 def _ptr(t):

@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include "common.cuh"
+#include "sched.cuh"
 
 using namespace skipffn;
 
@@ -12,13 +13,14 @@ struct skipffn_saved {
     size_t ws_bytes;
     int esize;
     // workspace carve-up (device)
-    int32_t *status, *idx, *pos;
-    void *Xk, *dOk, *G, *U, *H, *dG, *dU;
+    int32_t *status, *sk_flags, *idx, *pos;
+    void *sk_slots, *Xk, *dOk, *G, *U, *H, *dG, *dU;
     // state
     int64_t planned_N;     // tokens of the current index list, -1 if none
     int forwarded;
     const void *Wg, *Wu, *Wd;
     int launches[2];
+    int32_t sk_epoch;      // flag value of the latest tensor-core GEMM launch (never 0)
     // optional per-launch timing (CUDA events on the caller's stream)
     int profiling;
     cudaEvent_t ev[2 * SKIPFFN_PROFILE_SLOTS];
@@ -28,7 +30,7 @@ struct skipffn_saved {
 namespace {
 
 struct Layout {
-    size_t status, idx, pos, Xk, dOk, G, U, H, dG, dU, total;
+    size_t status, idx, pos, sk_slots, Xk, dOk, G, U, H, dG, dU, total;
 };
 
 bool valid_cfg(const skipffn_config *c)
@@ -44,9 +46,10 @@ Layout make_layout(const skipffn_config *c, int64_t max_tokens)
     const size_t es = c->dtype == SKIPFFN_BF16 ? 2 : 4;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
-    l.status = take(ST_WORDS * 4);
+    l.status = take((ST_WORDS + SK_FLAG_WORDS) * 4);   // status block, then the hand-over flags
     l.idx = take((size_t)cap * 4);
     l.pos = take((size_t)cap * 4);
+    l.sk_slots = take(c->dtype == SKIPFFN_BF16 ? (size_t)SK_MAX_CTAS * SK_SLOT_BYTES : 0);
     l.Xk = take((size_t)cap * c->C * es);
     l.dOk = take((size_t)cap * c->C * es);
     l.G = take((size_t)cap * c->I * es);
@@ -84,8 +87,11 @@ cudaError_t timed_launch(skipffn_saved *s, int slot, cudaStream_t st, F &&launch
     return cudaEventRecord(s->ev[2 * slot + 1], st);
 }
 
-cudaError_t run_gemm(skipffn_saved *s, int slot, int epi, const GemmArgs &g, cudaStream_t st)
+cudaError_t run_gemm(skipffn_saved *s, int slot, int epi, GemmArgs &g, cudaStream_t st)
 {
+    // every launch gets its own flag value, so flags left by earlier launches never match
+    if (++s->sk_epoch <= 0) s->sk_epoch = 1;
+    g.sk_epoch = s->sk_epoch;
     return timed_launch(s, slot, st, [&] {
         return use_umma(s) ? launch_umma_gemm(epi, g, st) : launch_simt_gemm(epi, s->cfg.dtype, g, st);
     });
@@ -97,6 +103,8 @@ GemmArgs base_args(const skipffn_saved *s)
     memset(&g, 0, sizeof(g));
     g.status = s->status;
     g.idx = s->idx;
+    g.sk_slots = s->sk_slots;
+    g.sk_flags = s->sk_flags;
     return g;
 }
 
@@ -146,6 +154,8 @@ skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config 
     s->esize = cfg->dtype == SKIPFFN_BF16 ? 2 : 4;
     char *w = (char *)workspace;
     s->status = (int32_t *)(w + l.status);
+    s->sk_flags = s->status + ST_WORDS;
+    s->sk_slots = w + l.sk_slots;
     s->idx = (int32_t *)(w + l.idx);
     s->pos = (int32_t *)(w + l.pos);
     s->Xk = w + l.Xk; s->dOk = w + l.dOk;
@@ -200,7 +210,7 @@ skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t 
     if (!skip_mask && !s->cfg.dense && N > 0) return SKIPFFN_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     // the status word is cleared together with the first plan of a handle
-    if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, ST_WORDS * 4, st) != cudaSuccess)
+    if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, st) != cudaSuccess)
         return SKIPFFN_ECUDA;
     s->launches[0] = 0;
     s->forwarded = 0;
@@ -227,7 +237,7 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     const int C = s->cfg.C, I = s->cfg.I;
     s->forwarded = 0;
     if (skip_mask || s->cfg.dense || N == 0) {
-        if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, ST_WORDS * 4, st) != cudaSuccess)
+        if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, st) != cudaSuccess)
             return SKIPFFN_ECUDA;
         s->launches[0] = 0;
         skipffn_status r = do_plan(s, skip_mask, N, 0, st);
@@ -363,6 +373,20 @@ skipffn_status skipffn_poll(skipffn_saved *s, void *stream, int32_t *site_out)
 int32_t skipffn_last_launches(const skipffn_saved *s, int32_t which)
 {
     return (s && (which == 0 || which == 1)) ? s->launches[which] : -1;
+}
+
+int32_t skipffn_schedule_segment(int32_t workers, int32_t tiles, int32_t k_blocks, int32_t split_k,
+                                 int32_t worker, int32_t i, int32_t *seg)
+{
+    if (workers <= 0 || tiles < 0 || k_blocks < 0 || worker < 0 || worker >= workers) return -1;
+    Sched sc;
+    sc.init(worker, workers, tiles, k_blocks, split_k);
+    const int n = sc.count();
+    if (seg && i >= 0 && i < n) {
+        const Seg g = sc.get(i);
+        seg[0] = g.tile; seg[1] = g.kb0; seg[2] = g.kb1; seg[3] = g.partial; seg[4] = g.src_lo;
+    }
+    return n;
 }
 
 double skipffn_flops(const skipffn_config *cfg, int64_t n_kept)

@@ -15,7 +15,15 @@ enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_WORDS = 64 };
 
 // Wait sites reported through the status word when a bounded wait gives up.
 enum : int { SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_TMEM_EMPTY = 3,
-             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5 };
+             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6 };
+
+// Split-K hand-over between CTAs of one tensor-core GEMM launch: a CTA that computes only part
+// of a tile's K range leaves its fp32 accumulator in its own slot of the workspace and raises one
+// flag per epilogue warp; the CTA that finishes the tile adds the slot to its accumulator.
+constexpr int SK_MAX_CTAS = 160;                    // slots (>= CTAs of a persistent launch)
+constexpr int SK_SLOT_BYTES = 128 * 256 * 4;        // one CTA's 128 x 256 fp32 accumulator
+constexpr int SK_FLAGS_PER_CTA = 8;                 // one per epilogue warp
+constexpr int SK_FLAG_WORDS = SK_MAX_CTAS * SK_FLAGS_PER_CTA;
 
 constexpr int ROW_PAD = 256;   // compacted buffers are zero-padded to this many rows past Nk
 
@@ -68,6 +76,10 @@ struct GemmArgs {
     int64_t ldo;                // leading dimension of outputs
     int32_t accumulate;         // DW epilogue: add to the destination
     int32_t out_fp32;           // DW epilogue: destination is float
+    // split-K hand-over (tensor-core path): slots, flags and this launch's flag value
+    void *sk_slots;
+    int32_t *sk_flags;
+    int32_t sk_epoch;
 };
 
 enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_DX = 4 };

@@ -25,12 +25,25 @@
 //               fills the other, apply the fused epilogue, write global memory
 //
 // The kept-token count Nk lives in device memory, so tile counts are derived on the device and no
-// host synchronisation sits between mask compaction and the GEMMs.  Every mbarrier wait is
-// bounded: on expiry the CTA records SKIPFFN_ETIMEOUT plus a site code and leaves normally.
+// host synchronisation sits between mask compaction and the GEMMs.  Every wait (mbarrier or
+// hand-over flag) is bounded: on expiry the CTA records SKIPFFN_ETIMEOUT plus a site code and
+// leaves normally.
+//
+// Work distribution.  A launch has T output tiles of KB K-blocks each and W tile workers (CTAs or
+// CTA pairs, all co-resident).  Whole waves of W tiles are handed out tile by tile; the tiles of
+// the last one-to-two waves (T mod W of them, plus W more when there are that many) are instead
+// cut along K into W equal, contiguous runs of K-blocks, one per worker, so that every worker
+// carries the same number of K-blocks whatever T mod W is.  A run that stops short of its last
+// tile's final K-block leaves that tile's fp32 partial accumulator in the worker's slot of the
+// workspace (each worker has at most one such run and processes it first); the worker whose run
+// contains the tile's final K-block adds the slots of its predecessors, in a fixed order, and
+// runs the epilogue.  The summation order depends only on the shapes, so results are
+// reproducible from run to run.
 #include <cuda.h>
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "sched.cuh"
 
 namespace skipffn {
 
@@ -112,6 +125,34 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status, site);
+}
+
+// Bounded wait of one warp for a hand-over flag written by another CTA of this launch.
+__device__ __noinline__ bool flag_wait(const int32_t *flag, int32_t want, int lane,
+                                       volatile int *abort_flag, int32_t *status)
+{
+    int ok = 1;
+    if (lane == 0) {
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            int32_t v;
+            asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+            if (v == want) break;
+            if ((it & 0x3f) == 0) {
+                if (*abort_flag) { ok = 0; break; }
+                if (t0 == 0) t0 = globaltimer_ns();
+                else if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+                    *abort_flag = 1;
+                    if (atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_ETIMEOUT) == 0)
+                        status[ST_SITE] = SITE_EPI_PARTIAL;
+                    ok = 0;
+                    break;
+                }
+            }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1,
@@ -284,6 +325,11 @@ struct UmmaParams {
     const void *in0, *in1;
     int64_t ldo;
     int32_t accumulate, out_fp32;
+    float4 *sk_slots;                // per-CTA partial-accumulator slots
+    int32_t *sk_flags;               // SK_FLAGS_PER_CTA flags per slot
+    int32_t sk_epoch;                // flag value of this launch
+    int32_t streamk;                 // 0: whole tiles only; else the least number of K-blocks per worker
+                                     // that cutting the last waves along K must save to be used
 };
 
 struct alignas(8) SmemCtl {
@@ -313,26 +359,6 @@ __device__ __forceinline__ void fast_swiglu_bwd(float dh, float g, float u, floa
     float s = fast_sigmoid(g);
     du = dh * (g * s);
     dg = dh * u * (s * (1.0f + g * (1.0f - s)));
-}
-
-// Tile width (accumulator columns) for this launch.  With few M tiles the tile count rarely fills
-// a whole number of waves of the persistent grid; narrower tiles trade MMA width for fewer idle
-// SMs in the last wave.  Cost model: waves x (MMA columns + B columns loaded, in 64-wide slabs).
-// `grid` = number of tile workers (CTAs, or CTA pairs); `split` = CTAs sharing the B tile.
-__device__ __forceinline__ int choose_bn(int num_m, int N, int grid, int force_bn, int split)
-{
-    if (force_bn > 0) return force_bn;
-    if (force_bn == 0) return BN;
-    int best = BN;
-    long best_cost = -1;
-    for (int bn = BN; bn >= 128; bn -= 16 * split) {
-        const int num_n = (N + bn - 1) / bn;
-        const long tiles = (long)num_m * num_n;
-        const long waves = (tiles + grid - 1) / grid;
-        const long cost = waves * (bn + 64 * split * ((bn / split + 63) / 64) + 32);
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
-    }
-    return best;
 }
 
 // Epilogue staging.  A warp owns 32 accumulator rows (one per lane).  For a 32-column bf16 chunk
@@ -422,14 +448,24 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
     const int num_m = (M + TILE_M - 1) / TILE_M;
-    // accumulator columns per tile; gate and up halves share a tile, so its output is half as wide
-    const int bn = GATEUP ? BN : choose_bn(num_m, p.N, num_workers, p.force_bn, SPLIT);
+    // accumulator columns per tile (256 unless overridden); gate and up halves share a tile, so its
+    // output is half as wide
+    const int bn = (GATEUP || p.force_bn <= 0) ? BN : p.force_bn;
     const int n_tile = GATEUP ? BN / 2 : bn;
     const int num_n = (p.N + n_tile - 1) / n_tile;
     const int num_tiles = num_m * num_n;
     const int kb_per_seg = (K + BK - 1) / BK;
     const int num_kb = kb_per_seg * p.segments;
     const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
+    Sched sched;
+    // Cutting the last waves costs every worker about two extra epilogues (one hand-over, one
+    // finish with the slot added); it pays when the idle time it removes, (W - T mod W) / W of a
+    // tile's main loop, is longer than that.
+    const int rem_tiles = num_tiles % num_workers;
+    const bool split_k = p.streamk > 0 && rem_tiles != 0 &&
+                         (long long)(num_workers - rem_tiles) * num_kb >= (long long)p.streamk * num_workers;
+    sched.init(worker, num_workers, num_tiles, num_kb, split_k);
+    const int num_segs = sched.count();
     const int bn_cta = bn / SPLIT;         // B rows (tile columns) this CTA stages
     const int b_slabs = (bn_cta + 63) / 64;
     const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
@@ -469,47 +505,53 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t stage_tx = SPLIT * (A_BYTES + b_slabs * CHUNK_BYTES);
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
+            // TMA loads of one K-block of one run into ring stage `stage`
+            auto issue = [&](const Seg &sg, int kb) {
+                const int tile = sg.tile;
                 const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
                 const int n0 = (tile / num_m) * n_tile;
                 const int nb0 = GATEUP ? n0 : n0 + (int)rank * bn_cta;   // first B row of this CTA
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const int seg = kb >= kb_per_seg ? 1 : 0;
+                const int k0 = (kb - seg * kb_per_seg) * BK;
+                const CUtensorMap *mA = seg ? &tmA2 : &tmA;
+                const CUtensorMap *mB = seg ? &tmB2 : &tmB;
+                const uint32_t own_bar = smem_u32(&ctl->full[stage]);
+                const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
+                const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                auto load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1) {
+                    if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar);
+                    else tma_load_2d(dst, map, c0, c1, bar);
+                };
+                if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
+                if (A_MN) {
+#pragma unroll
+                    for (int j = 0; j < BM / 64; ++j) load(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0);
+                } else {
+                    load(sa, mA, k0, m0);
+                }
+                if (B_MN) {          // 64-column slabs of BK rows
+                    for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, nb0 + 64 * j, k0);
+                } else if (GATEUP && PAIR) {   // leader stages the 128 gate rows, its peer the up rows
+#pragma unroll
+                    for (int j = 0; j < 2; ++j)
+                        load(sb + j * CHUNK_BYTES, rank == 0 ? &tmB : &tmB2, k0, n0 + 64 * j);
+                } else if (GATEUP) { // 128 gate rows, then 128 up rows, in 64-row pieces
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        load(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j);
+                        load(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j);
+                    }
+                } else {             // 64-row pieces of a K-major tile are contiguous in smem
+                    for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
+                }
+            };
+            for (int si = 0; ok && si < num_segs; ++si) {
+                const Seg sg = sched.get(si);
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
                     ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status,
                                    SITE_PRODUCER_EMPTY);
                     if (!ok) break;
-                    const int seg = kb >= kb_per_seg ? 1 : 0;
-                    const int k0 = (kb - seg * kb_per_seg) * BK;
-                    const CUtensorMap *mA = seg ? &tmA2 : &tmA;
-                    const CUtensorMap *mB = seg ? &tmB2 : &tmB;
-                    const uint32_t own_bar = smem_u32(&ctl->full[stage]);
-                    const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
-                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    auto load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1) {
-                        if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar);
-                        else tma_load_2d(dst, map, c0, c1, bar);
-                    };
-                    if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
-                    if (A_MN) {
-#pragma unroll
-                        for (int j = 0; j < BM / 64; ++j) load(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0);
-                    } else {
-                        load(sa, mA, k0, m0);
-                    }
-                    if (B_MN) {          // 64-column slabs of BK rows
-                        for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, nb0 + 64 * j, k0);
-                    } else if (GATEUP && PAIR) {   // leader stages the 128 gate rows, its peer the up rows
-#pragma unroll
-                        for (int j = 0; j < 2; ++j)
-                            load(sb + j * CHUNK_BYTES, rank == 0 ? &tmB : &tmB2, k0, n0 + 64 * j);
-                    } else if (GATEUP) { // 128 gate rows, then 128 up rows, in 64-row pieces
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            load(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j);
-                            load(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j);
-                        }
-                    } else {             // 64-row pieces of a K-major tile are contiguous in smem
-                        for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
-                    }
+                    issue(sg, kb);
                     if (++stage == nst) { stage = 0; phase ^= 1; }
                 }
             }
@@ -520,13 +562,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, TILE_M, bn);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
+            for (int si = 0; ok && si < num_segs; ++si) {
+                const Seg sg = sched.get(si);
                 ok = mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1, abort_flag, p.status,
                                SITE_MMA_TMEM_EMPTY);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
                     ok = mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, p.status,
                                    SITE_MMA_FULL);
                     if (!ok) break;
@@ -538,8 +581,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                                  : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
                         const uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
                                                  : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0);
-                        else umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
+                        const uint32_t accumulate = (kb != sg.kb0 || k != 0);   // first MMA of a run overwrites
+                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                        else umma_bf16(d_tmem, da, db, idesc, accumulate);
                     }
                     // the stage is reusable (in both CTAs) once these MMAs retire
                     if (PAIR) umma_commit_pair(smem_u32(&ctl->empty[stage]));
@@ -566,8 +610,48 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         bool ok = true;
         // accumulators are handed back on the leader's barrier, which its MMA warp waits on
         const uint32_t empty_bar0 = smem_u32(&ctl->tmem_empty[0]);
-        for (int tile = worker; ok && tile < num_tiles; tile += num_workers) {
+        // hand-over slots: a warp reads back exactly the words the same warp of the producing CTA wrote
+        const int my_slot = (int)blockIdx.x;
+        auto slot_ptr = [&](int cta_slot, int j) {
+            return p.sk_slots + (size_t)cta_slot * (SK_SLOT_BYTES / 16) + ((size_t)(ew * 4 + j) * 8) * 32 + lane;
+        };
+        for (int si = 0; ok && si < num_segs; ++si) {
+            const Seg sg = sched.get(si);
+            const int tile = sg.tile;
             const int m0 = (tile % num_m) * TILE_M + (int)rank * BM, n0 = (tile / num_m) * n_tile;
+            if (sg.partial) {
+                // ---- this run ends before the tile does: park the raw accumulator in this CTA's slot
+                ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
+                               SITE_EPI_TMEM_FULL);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
+#pragma unroll 1
+                for (int col = half * 32, j = 0; col < bn; col += 64, ++j) {
+                    uint32_t r[32];
+                    tmem_ld32(t_acc + col, r);
+                    tmem_ld_wait();
+                    float4 *dst = slot_ptr(my_slot, j);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        __stcg(dst + v * 32, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                         __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(p.sk_flags + my_slot * SK_FLAGS_PER_CTA + ew),
+                                 "r"(p.sk_epoch)
+                                 : "memory");
+                    const uint32_t bar = empty_bar0 + acc * 8;
+                    if (PAIR) mbar_arrive_cluster(mapa_rank(bar, 0));
+                    else mbar_arrive(bar);
+                }
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                continue;
+            }
+            const bool add_slots = sg.kb0 > 0;
             const int m = m0 + row_in_tile;
             const int n_end = min(n0 + n_tile, p.N);
             const bool row_valid = m < M;
@@ -597,6 +681,15 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 tc_fence_after();
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
+            if (add_slots) {
+                // the rest of this tile's K range sits in the slots of workers src_lo .. worker-1
+                for (int q = sg.src_lo; ok && q < worker; ++q) {
+                    if (sched.bound(q + 1) == sched.bound(q)) continue;   // that worker had no run
+                    ok = flag_wait(p.sk_flags + (q * SPLIT + (int)rank) * SK_FLAGS_PER_CTA + ew, p.sk_epoch,
+                                   lane, abort_flag, p.status);
+                }
+                if (!ok) break;
+            }
 
 #pragma unroll 1
             for (int n = n0 + half * 32; n < n_end; n += 64) {
@@ -614,6 +707,32 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 for (int v = 0; v < 4; ++v) { ca[v] = pa[v]; cb[v] = pb[v]; }
                 if (n + 64 < n_end) prefetch(n + 64);
                 if (!zero_acc) tmem_ld_wait();
+                if (add_slots) {
+                    const int j = col >> 6;   // this warp's j-th 32-column chunk of the accumulator
+                    for (int q = sg.src_lo; q < worker; ++q) {
+                        if (sched.bound(q + 1) == sched.bound(q)) continue;
+                        const float4 *src = slot_ptr(q * SPLIT + (int)rank, j);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const float4 a = __ldcg(src + v * 32);
+                            r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + a.x);
+                            r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + a.y);
+                            r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + a.z);
+                            r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + a.w);
+                        }
+                        if (GATEUP) {   // the up half of the accumulator: columns 128 + col
+                            const float4 *src2 = slot_ptr(q * SPLIT + (int)rank, j + 2);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) {
+                                const float4 a = __ldcg(src2 + v * 32);
+                                r2[GATEUP ? 4 * v : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v : 0]) + a.x);
+                                r2[GATEUP ? 4 * v + 1 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 1 : 0]) + a.y);
+                                r2[GATEUP ? 4 * v + 2 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 2 : 0]) + a.z);
+                                r2[GATEUP ? 4 * v + 3 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 3 : 0]) + a.w);
+                            }
+                        }
+                    }
+                }
                 const int valid_slots = min(4, (n_end - n) / 8);
                 uint32_t w[16];
                 if (EPI == EPI_GATEUP) {
@@ -796,7 +915,10 @@ static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CU
         }
     }
     if (max_workers <= 0) return cudaErrorNotSupported;
-    const int workers = (int)(max_tiles < max_workers ? max_tiles : max_workers);
+    // `max_tiles` = upper bound of the work items the launch can be cut into (tiles, or groups of
+    // K-blocks when tiles are split along K); every worker has its own hand-over slot
+    int workers = (int)(max_tiles < max_workers ? max_tiles : max_workers);
+    if (workers > SK_MAX_CTAS / (PAIR ? 2 : 1)) workers = SK_MAX_CTAS / (PAIR ? 2 : 1);
     if (workers <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
@@ -867,20 +989,31 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
     p.out0 = g.out0; p.out1 = g.out1; p.out2 = g.out2;
     p.in0 = g.in0; p.in1 = g.in1;
     p.ldo = g.ldo; p.accumulate = g.accumulate; p.out_fp32 = g.out_fp32;
+    p.sk_slots = (float4 *)g.sk_slots;
+    p.sk_flags = g.sk_flags;
+    p.sk_epoch = g.sk_epoch;
+    // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
+    static const int sk_threshold[5] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40};
+    p.streamk = (g.sk_slots && g.sk_flags) ? sk_threshold[epi] : 0;
+    if (const char *e = getenv("SKIPFFN_STREAMK")) { int v = atoi(e); if (v >= 0) p.streamk = v; }
 
     // SM pairs by default; SKIPFFN_SINGLE_CTA=1 (or a device that cannot co-schedule pairs) selects
     // the one-CTA-per-tile shape
     static int single = -1;
     if (single < 0) { const char *e = getenv("SKIPFFN_SINGLE_CTA"); single = (e && atoi(e) != 0) ? 1 : 0; }
-    const int n_tile = 128;   // narrowest tile the kernel may choose
+    const int n_tile = gateup ? BN / 2 : (p.force_bn > 0 ? p.force_bn : BN);   // output columns per tile
     const int64_t n_tiles = ((int64_t)g.N + n_tile - 1) / n_tile;
+    // with K splitting a tile can be shared by several workers: allow one worker per 4 K-blocks
+    const int64_t kb = ((int64_t)g.K + BK - 1) / BK * p.segments;
+    const int64_t per_tile = p.streamk ? (kb >= 8 ? kb / 4 : 1) : 1;
     if (!single) {
-        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + 2 * BM - 1) / (2 * BM) * n_tiles, s);
+        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, p,
+                                       ((int64_t)g.M + 2 * BM - 1) / (2 * BM) * n_tiles * per_tile, s);
         if (e != cudaErrorNotSupported) return e;
         (void)cudaGetLastError();
         single = 1;
     }
-    return dispatch<false>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + BM - 1) / BM * n_tiles, s);
+    return dispatch<false>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + BM - 1) / BM * n_tiles * per_tile, s);
 }
 
 }  // namespace skipffn

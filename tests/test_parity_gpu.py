@@ -103,6 +103,22 @@ def test_every_tile_width(tile_n, monkeypatch):
     _compare(w, run(w), _oracle_all(w))
 
 
+@pytest.mark.parametrize("min_saving", [0, 1])
+@pytest.mark.parametrize("case", ["tiny", "ragged", "wide"])
+def test_k_split_schedule_forced_on_and_off(min_saving, case, monkeypatch):
+    # SKIPFFN_STREAMK = least K-blocks per worker that cutting the last waves along K must save:
+    # 1 cuts whenever the tile count is not a multiple of the worker count (several hand-overs per
+    # tile on these small shapes), 0 never cuts.  Both must match the oracle.
+    monkeypatch.setenv("SKIPFFN_STREAMK", str(min_saving))
+    if case == "tiny":
+        w = wl.config1(dtype="bf16")
+    elif case == "ragged":
+        w = wl.small_case(23, "bf16", 576, 1000, 3, 20, 200, 0.6)
+    else:   # long reductions: I = 4096 gives 64 K-blocks for the down projection, 128 for dX
+        w = wl.small_case(25, "bf16", 256, 4096, 2, 16, 200, 0.5)
+    _compare(w, run(w), _oracle_all(w))
+
+
 def test_contiguous_span_layout():
     # the paper's layout: one contiguous skipped span per sequence
     w = wl.uniform_batch(2, "bf16", 256, 512, 4, 10, 150, 10, skip_ratio=0.8, contiguous_span=True)
