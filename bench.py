@@ -307,6 +307,8 @@ def run_ours(args):
     unit_flops = 2.0 * nk * C * I     # one GEMM "unit" of the path: 2 * Nk * C * I
     kernel_units = {"gateup": 2, "down": 1, "dh": 1, "dw_down": 1, "dw_gate": 1, "dw_up": 1, "dx": 2}
     kernels, roofline = {}, None
+    if prof and "dw_gate" not in prof and "dw_up" not in prof:
+        kernel_units["dw_down"] = 3     # one grouped launch computes all three weight gradients
     if prof:
         total = sum(prof.values())
         for name, kms in prof.items():
@@ -350,6 +352,68 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------ skip-ratio sweep
+def run_sweep(args):
+    """Skip-ratio sweep: visual skip fraction in {0, .25, .5, .75, .9, 1} at the LLaMA3-8B and
+    Vicuna-13B shapes (8 x 616 tokens), plus the in-library dense comparator on the same inputs.
+    One JSON line: per point kept tokens/s, TFLOP/s and time relative to dense."""
+    import torch
+    import paper_2503_21817_b200 as sk
+    torch.cuda.set_device(0)
+    pk = peaks()
+
+    def h_bf16(a):
+        return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).reshape(a.shape)
+
+    def time_ctx(ctx, x, mask, dout, W, bufs):
+        out, dx, dWg, dWu, dWd = bufs
+
+        def step():
+            ctx.forward(x, mask, W[0], W[1], W[2], out=out)
+            ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+        for _ in range(max(args.warmup, 3)):
+            step()
+        ctx.poll()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ctx.poll()
+        return e0.elapsed_time(e1) / args.steps
+
+    table = {}
+    for shape, (C, I) in wl.SWEEP_SHAPES.items():
+        base = wl.config2(seed=args.seed, skip_ratio=0.0, C=C, I=I)
+        weights = (base.W_gate, base.W_up, base.W_down)
+        W = [h_bf16(a).cuda() for a in weights]
+        x, dout = h_bf16(base.x).cuda(), h_bf16(base.dout).cuda()
+        bufs = [torch.empty_like(x), torch.empty_like(x)] + [torch.empty_like(t) for t in W]
+        dense = sk.SkipFFN(C, I, base.N, dense=True)
+        ms_dense = time_ctx(dense, x, torch.from_numpy(base.skip_mask).cuda(), dout, W, bufs)
+        del dense
+        ctx = sk.SkipFFN(C, I, base.N)
+        rows = []
+        for r in wl.SWEEP_RATIOS:
+            m = wl.config2(seed=args.seed, skip_ratio=r, C=8, I=8).skip_mask   # the mask depends on (seed, r) only
+            nk = int((m == 0).sum())
+            ms = time_ctx(ctx, x, torch.from_numpy(m).cuda(), dout, W, bufs)
+            tf = sk.skipffn_flops(C, I, nk) / (ms * 1e-3) / 1e12
+            rows.append({"skip_ratio": r, "kept_tokens": nk, "ms_per_step": ms, "kept_tokens_per_s": nk / (ms * 1e-3),
+                         "tflops": tf, "frac_of_measured_bf16_peak": tf / pk["bf16_tflops"],
+                         "time_vs_dense": ms / ms_dense, "kept_fraction": nk / base.N})
+        tf_dense = sk.skipffn_flops(C, I, base.N) / (ms_dense * 1e-3) / 1e12
+        table[shape] = {"C": C, "I": I, "tokens": base.N,
+                        "dense": {"ms_per_step": ms_dense, "tflops": tf_dense,
+                                  "frac_of_measured_bf16_peak": tf_dense / pk["bf16_tflops"]},
+                        "points": rows}
+        del ctx, W, x, dout, bufs
+    print(json.dumps({"sweep": "skip ratio", "steps": args.steps, "dtype": "bf16", "data": "synthetic",
+                      "peak_tflops": pk["bf16_tflops"], "peak_source": pk["source"], "shapes": table}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -365,8 +429,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile-only", action="store_true",
                     help="run warmup+steps steps and exit (launch sequence for an ncu capture)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="skip-ratio sweep at both shapes against the dense comparator (1 GPU)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

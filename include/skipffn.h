@@ -118,7 +118,9 @@ skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_ou
  * waits for those events and writes the elapsed milliseconds of each launch slot into
  * ms[SKIPFFN_PROFILE_SLOTS] (0 for slots that did not run): 0 mask compaction, 1 routing of x,
  * 2 gate/up GEMM, 3 down GEMM, 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate, 8 dW_up,
- * 9 dX GEMM. */
+ * 9 dX GEMM.  The tensor-core path computes the requested weight gradients in ONE grouped launch,
+ * whose time is reported in the slot of the first of them (6 when dW_down is requested) with the
+ * other two slots 0. */
 #define SKIPFFN_PROFILE_SLOTS 10
 skipffn_status skipffn_profile_enable(skipffn_saved *saved, int32_t on);
 skipffn_status skipffn_profile_read(skipffn_saved *saved, float *ms);

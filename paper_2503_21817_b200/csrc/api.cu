@@ -307,24 +307,36 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
     }
 
     // weight gradients: reductions over the kept-token axis (K = Nk, read on the device)
+    //   dWd[c, i] = sum_r dOk[r, c] H[r, i];  dWg[i, c] = sum_r dG[r, i] Xk[r, c];  dWu likewise with dU
     const int32_t kmax = (int32_t)N;
-    if (dW_down) {   // dWd[c, i] = sum_r dOk[r, c] H[r, i]
-        g = base_args(s);
-        g.A = s->dOk; g.lda_m = 1; g.lda_k = C; g.a_outer = s->cap;
-        g.B = s->H; g.ldb_n = 1; g.ldb_k = I; g.b_outer = s->cap;
-        g.M = C; g.N = I; g.K = kmax; g.k_from_nk = 1;
-        g.out0 = dW_down; g.ldo = I; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
-        if (run_gemm(s, SLOT_DW_DOWN, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    GemmArgs dw[3];
+    int dw_slot[3], n_dw = 0;
+    void *dw_dst[3] = {dW_down, dW_gate, dW_up};
+    for (int w = 0; w < 3; ++w) {
+        if (!dw_dst[w]) continue;
+        GemmArgs &q = dw[n_dw];
+        q = base_args(s);
+        if (w == 0) {
+            q.A = s->dOk; q.lda_k = C; q.B = s->H; q.ldb_k = I; q.M = C; q.N = I; q.ldo = I;
+        } else {
+            q.A = w == 1 ? s->dG : s->dU; q.lda_k = I; q.B = s->Xk; q.ldb_k = C; q.M = I; q.N = C; q.ldo = C;
+        }
+        q.lda_m = 1; q.ldb_n = 1; q.a_outer = s->cap; q.b_outer = s->cap;
+        q.K = kmax; q.k_from_nk = 1;
+        q.out0 = dw_dst[w]; q.accumulate = s->cfg.accumulate_dw;
+        q.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
+        dw_slot[n_dw++] = SLOT_DW_DOWN + w;
     }
-    for (int w = 0; w < 2; ++w) {   // dWg[i, c] = sum_r dG[r, i] Xk[r, c]; same for up with dU
-        void *dst = w == 0 ? dW_gate : dW_up;
-        if (!dst) continue;
-        g = base_args(s);
-        g.A = w == 0 ? s->dG : s->dU; g.lda_m = 1; g.lda_k = I; g.a_outer = s->cap;
-        g.B = s->Xk; g.ldb_n = 1; g.ldb_k = C; g.b_outer = s->cap;
-        g.M = I; g.N = C; g.K = kmax; g.k_from_nk = 1;
-        g.out0 = dst; g.ldo = C; g.accumulate = s->cfg.accumulate_dw; g.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
-        if (run_gemm(s, w == 0 ? SLOT_DW_GATE : SLOT_DW_UP, EPI_DW, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (use_umma(s) && n_dw > 1) {
+        // one grouped launch: the problems are independent, and together their tiles fill the
+        // persistent grid's waves better than one launch each; timed under the first one's slot
+        if (++s->sk_epoch <= 0) s->sk_epoch = 1;
+        for (int i = 0; i < n_dw; ++i) dw[i].sk_epoch = s->sk_epoch;
+        if (timed_launch(s, dw_slot[0], st, [&] { return launch_umma_dw_group(dw, n_dw, st); }) != cudaSuccess)
+            return SKIPFFN_ECUDA;
+    } else {
+        for (int i = 0; i < n_dw; ++i)
+            if (run_gemm(s, dw_slot[i], EPI_DW, dw[i], st) != cudaSuccess) return SKIPFFN_ECUDA;
     }
 
     if (N > 0) {   // dx[idx[r]] = dOk[r] + dG Wg + dU Wu

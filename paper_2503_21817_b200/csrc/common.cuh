@@ -92,5 +92,7 @@ cudaError_t launch_route(const RouteArgs &a, cudaStream_t s);
 cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
 // umma.cu (bf16 only)
 cudaError_t launch_umma_gemm(int epi, const GemmArgs &a, cudaStream_t s);
+// up to three weight-gradient problems (same K; problems 1 and 2 share B) in one launch
+cudaError_t launch_umma_dw_group(const GemmArgs *gs, int n, cudaStream_t s);
 
 }  // namespace skipffn

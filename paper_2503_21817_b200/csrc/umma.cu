@@ -328,6 +328,12 @@ struct UmmaParams {
     float4 *sk_slots;                // per-CTA partial-accumulator slots
     int32_t *sk_flags;               // SK_FLAGS_PER_CTA flags per slot
     int32_t sk_epoch;                // flag value of this launch
+    // grouped launch (weight gradients): up to three independent problems sharing K; problem g has
+    // extents gM[g] x gN[g], operands (tmA, tmB) / (tmA2, tmB2) / (tmA3, tmB2), output gout[g]
+    int32_t groups;
+    int32_t gM[3], gN[3];
+    void *gout[3];
+    int64_t gldo[3];
     int32_t streamk;                 // 0: whole tiles only; else the least number of K-blocks per worker
                                      // that cutting the last waves along K must save to be used
 };
@@ -426,7 +432,7 @@ template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
-            const UmmaParams p)
+            const __grid_constant__ CUtensorMap tmA3, const UmmaParams p)
 {
     constexpr bool GATEUP = (EPI == EPI_GATEUP);
     constexpr int STAGES = Shape<PAIR>::STAGES;
@@ -447,13 +453,32 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int nk = p.status[ST_NK];
     const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
-    const int num_m = (M + TILE_M - 1) / TILE_M;
     // accumulator columns per tile (256 unless overridden); gate and up halves share a tile, so its
     // output is half as wide
     const int bn = (GATEUP || p.force_bn <= 0) ? BN : p.force_bn;
     const int n_tile = GATEUP ? BN / 2 : bn;
-    const int num_n = (p.N + n_tile - 1) / n_tile;
-    const int num_tiles = num_m * num_n;
+    // tiles of problem g: ids [g_first[g], g_first[g+1]), the row-tile index running fastest
+    const int groups = (EPI == EPI_DW) ? p.groups : 1;
+    int g_m[3], g_n[3], g_num_m[3], g_first[4];
+    g_first[0] = 0;
+#pragma unroll
+    for (int g = 0; g < 3; ++g) {
+        g_m[g] = g < groups ? ((EPI == EPI_DW) ? p.gM[g] : M) : 0;
+        g_n[g] = g < groups ? ((EPI == EPI_DW) ? p.gN[g] : p.N) : 0;
+        g_num_m[g] = (g_m[g] + TILE_M - 1) / TILE_M;
+        g_first[g + 1] = g_first[g] + g_num_m[g] * ((g_n[g] + n_tile - 1) / n_tile);
+    }
+    const int num_tiles = g_first[3];
+    auto pick = [](const int (&a)[3], int g) { return g == 2 ? a[2] : (g == 1 ? a[1] : a[0]); };
+    struct TileLoc { int g, m0, n0; };
+    auto locate = [&](int tile) {
+        TileLoc t;
+        t.g = (EPI == EPI_DW) ? (tile >= g_first[2] ? 2 : (tile >= g_first[1] ? 1 : 0)) : 0;
+        const int local = tile - (t.g == 2 ? g_first[2] : (t.g == 1 ? g_first[1] : 0)), nm = pick(g_num_m, t.g);
+        t.m0 = (local % nm) * TILE_M;
+        t.n0 = (local / nm) * n_tile;
+        return t;
+    };
     const int kb_per_seg = (K + BK - 1) / BK;
     const int num_kb = kb_per_seg * p.segments;
     const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
@@ -499,8 +524,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0 && !zero_acc) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmB);
-            if (GATEUP || p.segments == 2) prefetch_tmap(&tmB2);
-            if (p.segments == 2) prefetch_tmap(&tmA2);
+            if (GATEUP || p.segments == 2 || groups > 1) prefetch_tmap(&tmB2);
+            if (p.segments == 2 || groups > 1) prefetch_tmap(&tmA2);
+            if (groups > 2) prefetch_tmap(&tmA3);
             // bytes landing on the (leader's) full barrier per stage, from every CTA of the tile
             const uint32_t stage_tx = SPLIT * (A_BYTES + b_slabs * CHUNK_BYTES);
             uint32_t stage = 0, phase = 0;
@@ -508,13 +534,13 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             // TMA loads of one K-block of one run into ring stage `stage`
             auto issue = [&](const Seg &sg, int kb) {
                 const int tile = sg.tile;
-                const int m0 = (tile % num_m) * TILE_M + (int)rank * BM;
-                const int n0 = (tile / num_m) * n_tile;
+                const TileLoc tl = locate(tile);
+                const int m0 = tl.m0 + (int)rank * BM, n0 = tl.n0;
                 const int nb0 = GATEUP ? n0 : n0 + (int)rank * bn_cta;   // first B row of this CTA
                 const int seg = kb >= kb_per_seg ? 1 : 0;
                 const int k0 = (kb - seg * kb_per_seg) * BK;
-                const CUtensorMap *mA = seg ? &tmA2 : &tmA;
-                const CUtensorMap *mB = seg ? &tmB2 : &tmB;
+                const CUtensorMap *mA = tl.g == 2 ? &tmA3 : ((tl.g == 1 || seg) ? &tmA2 : &tmA);
+                const CUtensorMap *mB = (tl.g >= 1 || seg) ? &tmB2 : &tmB;
                 const uint32_t own_bar = smem_u32(&ctl->full[stage]);
                 const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
                 const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -618,7 +644,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int si = 0; ok && si < num_segs; ++si) {
             const Seg sg = sched.get(si);
             const int tile = sg.tile;
-            const int m0 = (tile % num_m) * TILE_M + (int)rank * BM, n0 = (tile / num_m) * n_tile;
+            const TileLoc tl = locate(tile);
+            const int m0 = tl.m0 + (int)rank * BM, n0 = tl.n0;
             if (sg.partial) {
                 // ---- this run ends before the tile does: park the raw accumulator in this CTA's slot
                 ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
@@ -653,8 +680,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             const bool add_slots = sg.kb0 > 0;
             const int m = m0 + row_in_tile;
-            const int n_end = min(n0 + n_tile, p.N);
-            const bool row_valid = m < M;
+            const int n_end = min(n0 + n_tile, pick(g_n, tl.g));
+            const bool row_valid = m < pick(g_m, tl.g);
             int64_t tok = 0;
             if ((EPI == EPI_DOWN || EPI == EPI_DX) && row_valid) tok = p.idx[m];
             // prefetch of the per-row epilogue inputs of the first chunk (overlaps the accumulator wait)
@@ -789,8 +816,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     store_rows_64B(sbuf, lane, w, (char *)((bf16 *)p.out0 + o), valid_slots);
                     store_rows_64B(sbuf, lane, w2, (char *)((bf16 *)p.out1 + o), valid_slots);
                 } else {   // EPI_DW: weight-gradient tile, overwrite or accumulate
-                    const int64_t o = (int64_t)m * p.ldo + n;
-                    char *row = row_valid ? (char *)p.out0 + o * esz : nullptr;
+                    const int64_t o = (int64_t)m * p.gldo[tl.g] + n;
+                    char *row = row_valid ? (char *)p.gout[tl.g] + o * esz : nullptr;
                     if (p.out_fp32) {
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
@@ -888,8 +915,8 @@ static int g_num_sms = 0;
 // processed concurrently (CTAs, or CTA pairs).
 template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
-                            const CUtensorMap &b2, const UmmaParams &p, int64_t max_tiles,
-                            cudaStream_t s)
+                            const CUtensorMap &b2, const CUtensorMap &a3, const UmmaParams &p,
+                            int64_t max_tiles, cudaStream_t s)
 {
     constexpr int SMEM = Shape<PAIR>::SMEM_BYTES;
     static int max_workers = -1;   // -1 not yet queried; 0 unavailable
@@ -929,19 +956,20 @@ static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CU
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = PAIR ? 2 : 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, a, b, a2, b2, p);
+    return cudaLaunchKernelEx(&cfg, kern, a, b, a2, b2, a3, p);
 }
 
 template <bool PAIR>
 static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
-                            const CUtensorMap &b2, const UmmaParams &p, int64_t max_tiles, cudaStream_t s)
+                            const CUtensorMap &b2, const CUtensorMap &a3, const UmmaParams &p,
+                            int64_t max_tiles, cudaStream_t s)
 {
     switch (epi) {
-    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false, PAIR>(a, b, a2, b2, p, max_tiles, s);
-    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false, PAIR>(a, b, a2, b2, p, max_tiles, s);
-    case EPI_DH:     return launch_k<EPI_DH, false, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
-    case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
-    case EPI_DX:     return launch_k<EPI_DX, false, true, PAIR>(a, b, a2, b2, p, max_tiles, s);
+    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_DH:     return launch_k<EPI_DH, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_DX:     return launch_k<EPI_DX, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -949,8 +977,13 @@ static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b,
 // GemmArgs conventions: an operand with ld_k == 1 is K-major ([outer = M or N rows, inner = K]),
 // otherwise MN-major with ld_mn == 1 ([outer = K rows, inner = M or N]).  a_outer / b_outer give the
 // number of addressable rows of each array.
-cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
+// `n` > 1 (weight gradients only): up to three independent problems with the same K in one launch;
+// problems 1 and 2 share their B operand.
+static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStream_t s)
 {
+    if (n < 1 || n > 3 || (n > 1 && epi != EPI_DW)) return cudaErrorInvalidValue;
+    if (n == 3 && (gs[2].B != gs[1].B || gs[2].ldb_k != gs[1].ldb_k || gs[2].N != gs[1].N))
+        return cudaErrorInvalidValue;
     if (g_num_sms == 0) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
@@ -958,19 +991,26 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
         e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
     }
-    const bool a_mn = g.lda_k != 1, b_mn = g.ldb_k != 1;
+    const GemmArgs &g = gs[0];
     const bool gateup = epi == EPI_GATEUP;
-    CUtensorMap mA, mB, mA2, mB2;
+    CUtensorMap mA, mB, mA2, mB2, mA3;
     bool ok = true;
-    auto mk = [&](CUtensorMap *m, const void *base, bool mn, int64_t ld_mn, int64_t ld_k,
-                  int64_t mn_extent, int64_t outer_rows, int box_rows_kmajor) {
-        if (mn) return make_map(m, base, mn_extent, outer_rows, ld_k, BK);
-        return make_map(m, base, (int64_t)g.K, outer_rows, ld_mn, box_rows_kmajor);
+    auto mk = [&](CUtensorMap *m, const GemmArgs &q, const void *base, bool is_a) {
+        const int64_t ld_mn = is_a ? q.lda_m : q.ldb_n, ld_k = is_a ? q.lda_k : q.ldb_k;
+        const int64_t outer = is_a ? q.a_outer : q.b_outer;
+        if (ld_k != 1) return make_map(m, base, is_a ? q.M : q.N, outer, ld_k, BK);   // MN-major
+        return make_map(m, base, (int64_t)q.K, outer, ld_mn, is_a ? BM : 64);          // K-major
     };
-    ok &= mk(&mA, g.A, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM);
-    ok &= mk(&mB, g.B, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, 64);
-    if (g.A2) ok &= mk(&mA2, g.A2, a_mn, g.lda_m, g.lda_k, g.M, g.a_outer, BM); else mA2 = mA;
-    if (g.B2) ok &= mk(&mB2, g.B2, b_mn, g.ldb_n, g.ldb_k, g.N, g.b_outer, 64); else mB2 = mB;
+    ok &= mk(&mA, g, g.A, true);
+    ok &= mk(&mB, g, g.B, false);
+    if (n > 1) {
+        ok &= mk(&mA2, gs[1], gs[1].A, true);
+        ok &= mk(&mB2, gs[1], gs[1].B, false);
+    } else {
+        if (g.A2) ok &= mk(&mA2, g, g.A2, true); else mA2 = mA;
+        if (g.B2) ok &= mk(&mB2, g, g.B2, false); else mB2 = mB;
+    }
+    if (n > 2) ok &= mk(&mA3, gs[2], gs[2].A, true); else mA3 = mA;
     if (!ok) return cudaErrorInvalidValue;
 
     UmmaParams p;
@@ -989,6 +1029,12 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
     p.out0 = g.out0; p.out1 = g.out1; p.out2 = g.out2;
     p.in0 = g.in0; p.in1 = g.in1;
     p.ldo = g.ldo; p.accumulate = g.accumulate; p.out_fp32 = g.out_fp32;
+    p.groups = n;
+    for (int i = 0; i < 3; ++i) {
+        const GemmArgs &q = gs[i < n ? i : 0];
+        p.gM[i] = i < n ? q.M : 0; p.gN[i] = i < n ? q.N : 0;
+        p.gout[i] = q.out0; p.gldo[i] = q.ldo;
+    }
     p.sk_slots = (float4 *)g.sk_slots;
     p.sk_flags = g.sk_flags;
     p.sk_epoch = g.sk_epoch;
@@ -1002,18 +1048,32 @@ cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
     static int single = -1;
     if (single < 0) { const char *e = getenv("SKIPFFN_SINGLE_CTA"); single = (e && atoi(e) != 0) ? 1 : 0; }
     const int n_tile = gateup ? BN / 2 : (p.force_bn > 0 ? p.force_bn : BN);   // output columns per tile
-    const int64_t n_tiles = ((int64_t)g.N + n_tile - 1) / n_tile;
     // with K splitting a tile can be shared by several workers: allow one worker per 4 K-blocks
     const int64_t kb = ((int64_t)g.K + BK - 1) / BK * p.segments;
     const int64_t per_tile = p.streamk ? (kb >= 8 ? kb / 4 : 1) : 1;
+    auto max_items = [&](int tile_m) {
+        int64_t t = 0;
+        for (int i = 0; i < n; ++i)
+            t += (((int64_t)gs[i].M + tile_m - 1) / tile_m) * (((int64_t)gs[i].N + n_tile - 1) / n_tile);
+        return t * per_tile;
+    };
     if (!single) {
-        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, p,
-                                       ((int64_t)g.M + 2 * BM - 1) / (2 * BM) * n_tiles * per_tile, s);
+        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, mA3, p, max_items(2 * BM), s);
         if (e != cudaErrorNotSupported) return e;
         (void)cudaGetLastError();
         single = 1;
     }
-    return dispatch<false>(epi, mA, mB, mA2, mB2, p, ((int64_t)g.M + BM - 1) / BM * n_tiles * per_tile, s);
+    return dispatch<false>(epi, mA, mB, mA2, mB2, mA3, p, max_items(BM), s);
+}
+
+cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)
+{
+    return launch_problems(epi, &g, 1, s);
+}
+
+cudaError_t launch_umma_dw_group(const GemmArgs *gs, int n, cudaStream_t s)
+{
+    return launch_problems(EPI_DW, gs, n, s);
 }
 
 }  // namespace skipffn
