@@ -38,11 +38,11 @@ KERNEL_NAMES = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_
                 "dw_up", "dx"]
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each GEMM kernel at the
 # default workload, from the ncu captures summarised under profiles/; None until captured.
-NCU_TRAFFIC_BYTES = {"gateup": 368.7e6, "down": 235.7e6, "dh": 301.9e6, "dw_down": 129.0e6,
-                     "dw_gate": 170.3e6, "dw_up": 170.1e6, "dx": 451.0e6}
+NCU_TRAFFIC_BYTES = {"gateup": 365.1e6, "down": 367.6e6, "dh": 311.7e6, "dw_down": 545.2e6,
+                     "dx": 717.2e6, "route_x": 43.1e6, "route_dout": 42.3e6}
 # sha256 prefix of csrc/umma.cu when those counters were taken; once the kernel source differs the
 # counters no longer describe it and `traffic` is reported as null
-NCU_TRAFFIC_SOURCE_SHA = "faef05494660a744"
+NCU_TRAFFIC_SOURCE_SHA = "cd427f4d6c9a0960"
 
 
 def ncu_traffic(kernel):
@@ -313,6 +313,13 @@ def run_ours(args):
         total = sum(prof.values())
         for name, kms in prof.items():
             ent = {"ms": kms, "share": kms / total if total else None}
+            if name in ("route_x", "route_dout"):
+                # every row is read once and written once (kept rows compacted, skipped rows copied)
+                ent["gbs"] = (2.0 * N * C * 2 + 4.0 * N) / (kms * 1e-3) / 1e9
+                ent["frac_of_measured_hbm"] = ent["gbs"] / pk["hbm_gbs"]
+            if name == "compact":
+                ent["gbs"] = (N + 4.0 * N + 4.0 * nk) / (kms * 1e-3) / 1e9      # mask in; pos, idx out
+                ent["bound"] = "latency (one CTA)"
             if name in kernel_units:
                 ent["tflops"] = kernel_units[name] * unit_flops / (kms * 1e-3) / 1e12
                 ent["frac_of_measured_bf16_peak"] = ent["tflops"] / pk["bf16_tflops"]
@@ -323,7 +330,7 @@ def run_ours(args):
                     "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": gemms[top]["tflops"] / pk["bf16_tflops"],
                     "peak_source": pk["source"] + " (burst cuBLAS bf16)",
                     "traffic": ncu_traffic(top),
-                    "all_gemm_kernels": {"tflops": sum(kernel_units.values()) * unit_flops /
+                    "all_gemm_kernels": {"tflops": sum(kernel_units[k] for k in gemms) * unit_flops /
                                          (sum(v["ms"] for v in gemms.values()) * 1e-3) / 1e12}}
         roofline["all_gemm_kernels"]["frac"] = roofline["all_gemm_kernels"]["tflops"] / pk["bf16_tflops"]
 
