@@ -245,13 +245,51 @@ def run_ours(args):
         ctx.forward(x, mask, Wg, Wu, Wd, out=out)
         ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
 
+    # End-to-end leg: every step copies x, skip_mask and dout from pinned host memory and copies
+    # out and dx back.  Two sets of device buffers and three streams (host->device, compute,
+    # device->host) let step i+1's input copy and step i-1's result copy run under step i's
+    # kernels; events order each buffer's copy -> compute -> copy-back -> reuse.
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    s_comp = torch.cuda.current_stream(dev)
+    dbuf = [dict(x=torch.empty_like(x), mask=torch.empty_like(mask), dout=torch.empty_like(dout),
+                 out=torch.empty_like(x), dx=torch.empty_like(x),
+                 ready_in=torch.cuda.Event(), done=torch.cuda.Event(), copied_out=torch.cuda.Event())
+            for _ in range(2)]
+    e2e_count = [0]
+
     def step_e2e():
-        x.copy_(hx, non_blocking=True)
-        mask.copy_(hmask, non_blocking=True)
-        dout.copy_(hdout, non_blocking=True)
-        step()
-        hout.copy_(out, non_blocking=True)
-        hdx.copy_(dx, non_blocking=True)
+        b = dbuf[e2e_count[0] % 2]
+        first_use = e2e_count[0] < 2
+        e2e_count[0] += 1
+        with torch.cuda.stream(s_in):
+            if not first_use:
+                s_in.wait_event(b["done"])          # the step that last read these inputs has finished
+            b["x"].copy_(hx, non_blocking=True)
+            b["mask"].copy_(hmask, non_blocking=True)
+            b["dout"].copy_(hdout, non_blocking=True)
+            b["ready_in"].record(s_in)
+        s_comp.wait_event(b["ready_in"])
+        if not first_use:
+            s_comp.wait_event(b["copied_out"])      # its previous results are on the host
+        ctx.forward(b["x"], b["mask"], Wg, Wu, Wd, out=b["out"])
+        ctx.backward(b["dout"], dx=b["dx"], dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+        b["done"].record(s_comp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(b["done"])
+            hout.copy_(b["out"], non_blocking=True)
+            hdx.copy_(b["dx"], non_blocking=True)
+            b["copied_out"].record(s_out)
+
+    def timed_e2e(steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(s_in)                              # nothing is in flight: the first copy starts here
+        for _ in range(steps):
+            step_e2e()
+        s_out.wait_stream(s_comp)
+        e1.record(s_out)                             # after the last result has reached the host
+        barrier()
+        return e0.elapsed_time(e1)
 
     def barrier():
         torch.cuda.synchronize()
@@ -286,9 +324,9 @@ def run_ours(args):
     ctx.poll()
     launches_per_step = sum(ctx.launches())
 
-    for _ in range(2):
+    for _ in range(3):
         step_e2e()
-    ms_e2e, _, _ = timed(step_e2e, args.steps)
+    ms_e2e = timed_e2e(args.steps)
 
     # per-kernel durations: the same steps again with CUDA events recorded around every launch
     prof = ctx.profile(step, args.steps) if hasattr(ctx, "profile") else None
@@ -351,7 +389,8 @@ def run_ours(args):
             "frac_of_sustained_bf16_peak": (tflops / world / pk["bf16_tflops_sustained"]) if pk["bf16_tflops_sustained"] else None,
             "frac_of_nominal_bf16_peak": tflops / world / 2250.0,
             "e2e": {"value": value_e2e, "unit": UNIT,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_step_e2e},
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_step_e2e,
+                    "pipeline": "3 streams (H2D, compute, D2H), double-buffered device inputs and results"},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
             "kernels": kernels, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
@@ -421,6 +460,40 @@ def run_sweep(args):
                       "peak_tflops": pk["bf16_tflops"], "peak_source": pk["source"], "shapes": table}), flush=True)
 
 
+# ------------------------------------------------------------------------------ library yardstick
+def run_yardstick(args):
+    """Not part of the metric: times the vendor library's plain GEMMs (torch.matmul) on the five
+    contraction shapes of the path, same box, same timing method, for context beside the fused
+    kernels (which also write G, U, H, apply SiLU*mul / its derivative and scatter residual rows)."""
+    import torch
+    torch.cuda.set_device(0)
+    C, I = wl.SWEEP_SHAPES[args.shape]
+    nk = wl.config2(seed=args.seed, skip_ratio=args.skip_ratio, C=8, I=8).n_kept
+    bf, dev = torch.bfloat16, "cuda"
+    g = torch.Generator(device=dev).manual_seed(0)
+    rnd = lambda *sh: torch.randn(*sh, device=dev, dtype=bf, generator=g)
+    X, dO, H, dG, dGU = rnd(nk, C), rnd(nk, C), rnd(nk, I), rnd(nk, I), rnd(nk, 2 * I)
+    Wgu, Wd = rnd(2 * I, C), rnd(C, I)
+    cases = [("gateup", lambda: X @ Wgu.T, 2), ("down", lambda: H @ Wd.T, 1), ("dh", lambda: dO @ Wd, 1),
+             ("dw_down", lambda: dO.T @ H, 1), ("dw_gate", lambda: dG.T @ X, 1), ("dw_up", lambda: dG.T @ X, 1),
+             ("dx", lambda: dGU @ Wgu, 2)]
+    out = {}
+    for name, fn, units in cases:
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.steps
+        out[name] = {"ms": ms, "tflops": units * 2.0 * nk * C * I / (ms * 1e-3) / 1e12}
+    print(json.dumps({"yardstick": "torch.matmul bf16, plain GEMMs of the path's shapes", "kept_tokens": nk,
+                      "C": C, "I": I, "sum_ms": sum(v["ms"] for v in out.values()), "gemms": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -438,8 +511,12 @@ def main():
                     help="run warmup+steps steps and exit (launch sequence for an ncu capture)")
     ap.add_argument("--sweep", action="store_true",
                     help="skip-ratio sweep at both shapes against the dense comparator (1 GPU)")
+    ap.add_argument("--yardstick", action="store_true",
+                    help="time the vendor library's plain GEMMs on the path's shapes (context only)")
     args = ap.parse_args()
-    if args.sweep:
+    if args.yardstick:
+        run_yardstick(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
