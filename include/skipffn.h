@@ -102,6 +102,23 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *saved, void *dx
 skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
                                 const int32_t **nk_dev);
 
+/* Skip KV-cache (paper section 4.3, Eq. 7): after prefill the cache keeps only the keys / values of
+ * the retained tokens, K' = K \ K_skip, in their original order.  Uses the kept-row list of the
+ * last skipffn_plan / skipffn_forward on `saved` (N = its token count).
+ *   src : [planes, N, row_bytes] device bytes: any number of leading dimensions (layer, key/value)
+ *         flattened into `planes`, then the token axis, then one token's heads x head_dim values
+ *         (the packed "total tokens" layout); row_bytes a multiple of 16.
+ *   dst : [planes, dst_rows, row_bytes]; rows 0 .. min(Nk, dst_rows)-1 of every plane receive the
+ *         kept rows, byte for byte; other rows are not written.  Must not overlap src (EINVAL).
+ *   cu_seqlens / kept_cu_seqlens : optional DEVICE int32 arrays of n_seq+1 entries; when
+ *         kept_cu_seqlens is given it receives the sequence offsets of the pruned cache, i.e. the
+ *         number of kept tokens before each cu_seqlens[s].
+ * Enqueued on `stream`; Nk stays on the device. */
+skipffn_status skipffn_kv_compact(const skipffn_saved *saved, const void *src, void *dst,
+                                  int64_t planes, int64_t row_bytes, int64_t dst_rows,
+                                  const int32_t *cu_seqlens, int32_t n_seq,
+                                  int32_t *kept_cu_seqlens, void *stream);
+
 /* Device addresses of the compacted intermediates of the last forward / backward, each
  * [round_up(Nk,128), I] in cfg.dtype (rows >= Nk are zero): which = 0 G, 1 U, 2 H, 3 dG, 4 dU;
  * 5 = kept rows of x [.., C]; 6 = kept rows of dout [.., C]. */

@@ -48,6 +48,10 @@ def _load() -> ctypes.CDLL:
         lib.skipffn_oracle_dw_columns.restype = None
         lib.skipffn_oracle_dw_columns.argtypes = [dp, bp, dp, dp, dp, dp, i64, i64, i64, dp, i64,
                                                   dp, dp, dp]
+        lib.skipffn_oracle_kv_compact.restype = i64
+        lib.skipffn_oracle_kv_compact.argtypes = [bp, bp, i64, i64, i64, bp]
+        lib.skipffn_oracle_kept_cu_seqlens.restype = None
+        lib.skipffn_oracle_kept_cu_seqlens.argtypes = [bp, ctypes.c_void_p, i64, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -136,3 +140,28 @@ def dw_columns(x, skip_mask, W_gate, W_up, W_down, dout, cols: Sequence[int]):
     _load().skipffn_oracle_dw_columns(_p(x), _p(m), _p(wg), _p(wu), _p(wd), _p(do), N, C, I,
                                       _p(cc), cc.size, _p(a), _p(b), _p(c))
     return a, b, c
+
+
+def kv_compact(cache, skip_mask) -> np.ndarray:
+    """Skip KV-cache (Eq. 7): ``cache`` ``[planes, N, ...]`` (any dtype) without the rows of the
+    skipped tokens, ``[planes, n_kept, ...]``, original order, byte for byte."""
+    c = np.ascontiguousarray(cache)
+    m = _u8(skip_mask)
+    planes, N = c.shape[0], c.shape[1]
+    assert m.size == N
+    row_bytes = int(np.prod(c.shape[2:], dtype=np.int64)) * c.itemsize
+    nk = int(N - np.count_nonzero(m))
+    out = np.empty((planes, nk) + c.shape[2:], dtype=c.dtype)
+    got = _load().skipffn_oracle_kv_compact(_p(c.view(np.uint8).reshape(-1)), _p(m), planes, N, row_bytes,
+                                            _p(out.view(np.uint8).reshape(-1)))
+    assert got == nk
+    return out
+
+
+def kept_cu_seqlens(skip_mask, cu_seqlens) -> np.ndarray:
+    """Sequence offsets of the pruned cache: number of retained tokens before each offset."""
+    m = _u8(skip_mask)
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    out = np.empty_like(cu)
+    _load().skipffn_oracle_kept_cu_seqlens(_p(m), _p(cu), cu.size, _p(out))
+    return out

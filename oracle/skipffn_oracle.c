@@ -27,7 +27,8 @@
  * inputs, scalar closed form, W_gate = 0 / W_down = 0 identities, all-kept ==
  * dense FFN via a library matmul, all-skipped == input, central finite
  * differences for every gradient, linearity and homogeneity properties, and the
- * per-layer skip error of Eq. 8.
+ * per-layer skip error of Eq. 8.  Skip KV-cache: library boolean indexing, a set-difference
+ * restatement of Eq. 7 on tagged rows, and hand-written tiny cases.
  */
 #include <math.h>
 #include <stdint.h>
@@ -196,5 +197,41 @@ void skipffn_oracle_dw_columns(const double *x, const uint8_t *skip_mask, const 
                 ru[c] += du * xt[c];
             }
         }
+    }
+}
+
+/* Skip KV-cache (section 4.3, Eq. 7): the cache after prefill is the set difference
+ * K_cache \ K_skip (likewise V), i.e. the rows of the retained tokens in their original order.
+ * src: [planes, N, row_bytes] bytes; dst: [planes, n_kept, row_bytes], written densely.
+ * Returns n_kept.  Plain byte copies, one token at a time. */
+int64_t skipffn_oracle_kv_compact(const uint8_t *src, const uint8_t *skip_mask, int64_t planes,
+                                  int64_t N, int64_t row_bytes, uint8_t *dst)
+{
+    int64_t n_kept = 0;
+    for (int64_t t = 0; t < N; ++t)
+        if (skip_mask[t] == 0)
+            ++n_kept;
+    for (int64_t p = 0; p < planes; ++p) {
+        int64_t r = 0;
+        for (int64_t t = 0; t < N; ++t) {
+            if (skip_mask[t] != 0)
+                continue; /* a skipped token's key / value leaves the cache */
+            memcpy(dst + (p * n_kept + r) * row_bytes, src + (p * N + t) * row_bytes, (size_t)row_bytes);
+            ++r;
+        }
+    }
+    return n_kept;
+}
+
+/* Sequence offsets of the pruned cache: kept_cu[s] = number of retained tokens before cu[s]. */
+void skipffn_oracle_kept_cu_seqlens(const uint8_t *skip_mask, const int32_t *cu, int64_t n_entries,
+                                    int32_t *kept_cu)
+{
+    for (int64_t s = 0; s < n_entries; ++s) {
+        int32_t c = 0;
+        for (int64_t t = 0; t < cu[s]; ++t)
+            if (skip_mask[t] == 0)
+                ++c;
+        kept_cu[s] = c;
     }
 }

@@ -17,7 +17,7 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
            "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
-           "skipffn_compact_static", "skipffn_schedule_segment"]
+           "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_compact_static.argtypes = [vp, i64, vp, vp, vp]
     lib.skipffn_schedule_segment.restype = i32
     lib.skipffn_schedule_segment.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
+    lib.skipffn_kv_compact.restype = i32
+    lib.skipffn_kv_compact.argtypes = [vp, vp, vp, i64, i64, i64, vp, i32, vp, vp]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -270,6 +272,40 @@ class SkipFFN:
         if st != 0:
             raise SkipFFNError(st, "skipffn_backward")
         return dx, dW_gate, dW_up, dW_down
+
+    def kv_compact(self, src, dst=None, cu_seqlens=None):
+        """Skip KV-cache (``skipffn_kv_compact``, Eq. 7) with the current kept-row list.
+
+        ``src``: contiguous CUDA tensor ``[planes..., N, heads, head_dim]`` (4-D or more) or
+        ``[planes..., N, row]``; N must be the token count of the last plan / forward.  ``dst``
+        (default: a new tensor shaped like ``src``) receives the kept rows in the first Nk
+        positions of its token axis.  Returns ``(dst, kept_cu_seqlens)``; the second is an int32
+        CUDA tensor if ``cu_seqlens`` was given, else ``None``."""
+        torch = self._torch
+        if not src.is_cuda or not src.is_contiguous():
+            raise ValueError("src must be a contiguous CUDA tensor")
+        tok_axis = src.dim() - 3 if src.dim() >= 4 else src.dim() - 2
+        N = src.shape[tok_axis]
+        planes = 1
+        for d in src.shape[:tok_axis]:
+            planes *= d
+        row_bytes = src.element_size()
+        for d in src.shape[tok_axis + 1:]:
+            row_bytes *= d
+        if dst is None:
+            dst = torch.empty_like(src)
+        dst_rows = dst.shape[tok_axis]
+        cu_dev = new_cu = None
+        n_seq = 0
+        if cu_seqlens is not None:
+            cu_dev = torch.as_tensor([int(v) for v in cu_seqlens], dtype=torch.int32, device=self.device)
+            new_cu = torch.empty_like(cu_dev)
+            n_seq = cu_dev.numel() - 1
+        st = self.lib.skipffn_kv_compact(self._saved, _ptr(src), _ptr(dst), planes, row_bytes, dst_rows,
+                                         _ptr(cu_dev), n_seq, _ptr(new_cu), self._stream())
+        if st != 0:
+            raise SkipFFNError(st, "skipffn_kv_compact")
+        return dst, new_cu
 
     def poll(self):
         """Synchronise the stream and raise if a kernel reported a device-side problem."""

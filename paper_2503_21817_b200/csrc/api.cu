@@ -350,6 +350,31 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
     return SKIPFFN_OK;
 }
 
+skipffn_status skipffn_kv_compact(const skipffn_saved *s, const void *src, void *dst, int64_t planes,
+                                  int64_t row_bytes, int64_t dst_rows, const int32_t *cu_seqlens,
+                                  int32_t n_seq, int32_t *kept_cu_seqlens, void *stream)
+{
+    if (!s || s->planned_N < 0 || planes < 0 || row_bytes <= 0 || dst_rows < 0) return SKIPFFN_EINVAL;
+    if (row_bytes % 16) return SKIPFFN_EUNSUPPORTED;
+    const int64_t N = s->planned_N;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (planes > 0 && N > 0 && dst_rows > 0) {
+        if (!src || !dst || !aligned16(src) || !aligned16(dst)) return SKIPFFN_EINVAL;
+        // the gather runs in parallel over rows, so the two caches must not overlap
+        const char *a = (const char *)src, *b = (const char *)dst;
+        const int64_t src_bytes = planes * N * row_bytes, dst_bytes = planes * dst_rows * row_bytes;
+        if (a < b + dst_bytes && b < a + src_bytes) return SKIPFFN_EINVAL;
+        if (launch_kv_compact(src, dst, s->idx, s->status, planes, N, dst_rows, row_bytes, st) != cudaSuccess)
+            return SKIPFFN_ECUDA;
+    }
+    if (kept_cu_seqlens) {
+        if (!cu_seqlens || n_seq < 0) return SKIPFFN_EINVAL;
+        if (launch_kept_cu_seqlens(cu_seqlens, kept_cu_seqlens, n_seq + 1, s->idx, s->status, st) != cudaSuccess)
+            return SKIPFFN_ECUDA;
+    }
+    return SKIPFFN_OK;
+}
+
 skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev, const int32_t **nk_dev)
 {
     if (!s || s->planned_N < 0) return SKIPFFN_EINVAL;

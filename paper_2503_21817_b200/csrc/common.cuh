@@ -88,6 +88,12 @@ enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
                            int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs &a, cudaStream_t s);
+// kvcache.cu
+cudaError_t launch_kv_compact(const void *src, void *dst, const int32_t *idx, const int32_t *status,
+                              int64_t planes, int64_t N, int64_t dst_rows, int64_t row_bytes,
+                              cudaStream_t s);
+cudaError_t launch_kept_cu_seqlens(const int32_t *cu, int32_t *new_cu, int n, const int32_t *idx,
+                                   const int32_t *status, cudaStream_t s);
 // simt.cu
 cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
 // umma.cu (bf16 only)

@@ -101,7 +101,16 @@ k_route(const uint4 *__restrict__ src, uint4 *__restrict__ dst_compact,
         if (p >= 0) d = dst_compact + (int64_t)p * row_vecs;
         else if (copy_identity) d = dst_identity + u * row_vecs;
         else return;
-        for (int v = threadIdx.x; v < row_vecs; v += RT_THREADS) d[v] = s[v];
+        // four 16-byte loads in flight per thread before the first store; rows are read once
+        for (int v0 = threadIdx.x; v0 < row_vecs; v0 += 4 * RT_THREADS) {
+            uint4 t[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v0 + u * RT_THREADS < row_vecs) t[u] = __ldcs(s + v0 + u * RT_THREADS);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v0 + u * RT_THREADS < row_vecs) d[v0 + u * RT_THREADS] = t[u];
+        }
     } else {
         int nk = status[ST_NK];
         int64_t r = nk + (u - N);

@@ -278,3 +278,43 @@ def test_paper_table1_fixes_swiglu_shape():
     x, mask, wg, wu, wd, _ = _rand_case(2, 4, 14)
     assert wg.size + wu.size + wd.size == g["ffn_macs_per_token_coeff"] * 4 * 14
     oracle.forward(x, mask, wg, wu, wd)
+
+
+# ------------------------------------------------------------------ skip KV-cache (Eq. 7)
+def test_kv_compact_is_the_set_difference_in_order():
+    r = np.random.default_rng(7)
+    planes, N, heads, d = 3, 41, 2, 4
+    mask = (r.random(N) < 0.6).astype(np.uint8) * r.integers(1, 200, size=N).astype(np.uint8)
+    # tag every row with (plane, token) so that rows are distinguishable set elements
+    cache = np.zeros((planes, N, heads, d), dtype=np.float32)
+    cache[..., 0, 0] = np.arange(planes)[:, None]
+    cache[..., 0, 1] = np.arange(N)[None, :]
+    cache[..., 1, :] = r.normal(size=(planes, N, d))
+    out = oracle.kv_compact(cache, mask)
+    # library routine: boolean indexing
+    assert np.array_equal(out, cache[:, mask == 0])
+    # Eq. 7 as a set difference: the tokens present afterwards are exactly those not skipped
+    for p in range(planes):
+        present = [int(t) for t in out[p, :, 0, 1]]
+        assert set(present) == set(range(N)) - set(np.flatnonzero(mask).tolist())
+        assert present == sorted(present)                       # original order
+        assert np.all(out[p, :, 0, 0] == p)                     # no mixing across planes
+    # NaN payloads and negative zero survive a byte copy
+    cache[0, int(np.flatnonzero(mask == 0)[0]), 1, 0] = np.nan
+    cache[0, int(np.flatnonzero(mask == 0)[0]), 1, 1] = -0.0
+    out = oracle.kv_compact(cache, mask)
+    assert out.tobytes() == cache[:, mask == 0].tobytes()
+
+
+def test_kv_compact_hand_cases_and_offsets():
+    cache = np.arange(2 * 5 * 2, dtype=np.int16).reshape(2, 5, 2)
+    out = oracle.kv_compact(cache, [0, 1, 1, 0, 0])
+    assert out.tolist() == [[[0, 1], [6, 7], [8, 9]], [[10, 11], [16, 17], [18, 19]]]
+    assert oracle.kv_compact(cache, [1] * 5).shape == (2, 0, 2)
+    assert np.array_equal(oracle.kv_compact(cache, [0] * 5), cache)
+    # offsets: sequences [0,2) [2,5): one kept in the first, two in the second
+    assert oracle.kept_cu_seqlens([0, 1, 1, 0, 0], [0, 2, 5]).tolist() == [0, 1, 3]
+    w = wl.config4(seed=1, C=8, I=8, n_seq=5)
+    got = oracle.kept_cu_seqlens(w.skip_mask, w.cu_seqlens)
+    want = [int((w.skip_mask[:c] == 0).sum()) for c in w.cu_seqlens]
+    assert got.tolist() == want and got[-1] == w.n_kept
