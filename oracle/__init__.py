@@ -48,6 +48,11 @@ def _load() -> ctypes.CDLL:
         lib.skipffn_oracle_dw_columns.restype = None
         lib.skipffn_oracle_dw_columns.argtypes = [dp, bp, dp, dp, dp, dp, i64, i64, i64, dp, i64,
                                                   dp, dp, dp]
+        lib.skipffn_oracle_forward_prenorm.restype = None
+        lib.skipffn_oracle_forward_prenorm.argtypes = [dp, bp, dp, ctypes.c_double, dp, dp, dp, i64, i64, i64, dp]
+        lib.skipffn_oracle_backward_prenorm.restype = None
+        lib.skipffn_oracle_backward_prenorm.argtypes = [dp, bp, dp, ctypes.c_double, dp, dp, dp, dp, i64, i64, i64,
+                                                        dp, dp, dp, dp, dp]
         lib.skipffn_oracle_kv_compact.restype = i64
         lib.skipffn_oracle_kv_compact.argtypes = [bp, bp, i64, i64, i64, bp]
         lib.skipffn_oracle_kept_cu_seqlens.restype = None
@@ -165,3 +170,30 @@ def kept_cu_seqlens(skip_mask, cu_seqlens) -> np.ndarray:
     out = np.empty_like(cu)
     _load().skipffn_oracle_kept_cu_seqlens(_p(m), _p(cu), cu.size, _p(out))
     return out
+
+
+def forward_prenorm(x, skip_mask, gamma, eps, W_gate, W_up, W_down) -> np.ndarray:
+    """Pre-norm variant: ``x + FFN(RMSNorm(x) * gamma)`` on kept rows, ``x`` on skipped rows."""
+    x, g, wg, wu, wd, m = _f64(x), _f64(gamma), _f64(W_gate), _f64(W_up), _f64(W_down), _u8(skip_mask)
+    N, C = x.shape
+    I = wg.shape[0]
+    assert g.shape == (C,) and wg.shape == (I, C) and wu.shape == (I, C) and wd.shape == (C, I) and m.size == N
+    out = np.empty((N, C), dtype=np.float64)
+    _load().skipffn_oracle_forward_prenorm(_p(x), _p(m), _p(g), float(eps), _p(wg), _p(wu), _p(wd), N, C, I, _p(out))
+    return out
+
+
+def backward_prenorm(x, skip_mask, gamma, eps, W_gate, W_up, W_down, dout, need_dw: bool = True):
+    """``(dx, dgamma, dW_gate, dW_up, dW_down)`` of the pre-norm variant for the loss ``sum(dout * out)``."""
+    x, g, wg, wu, wd, m, do = (_f64(x), _f64(gamma), _f64(W_gate), _f64(W_up), _f64(W_down), _u8(skip_mask),
+                               _f64(dout))
+    N, C = x.shape
+    I = wg.shape[0]
+    dx = np.empty((N, C), dtype=np.float64)
+    dg = np.empty(C, dtype=np.float64)
+    dwg = np.empty((I, C), dtype=np.float64) if need_dw else None
+    dwu = np.empty((I, C), dtype=np.float64) if need_dw else None
+    dwd = np.empty((C, I), dtype=np.float64) if need_dw else None
+    _load().skipffn_oracle_backward_prenorm(_p(x), _p(m), _p(g), float(eps), _p(wg), _p(wu), _p(wd), _p(do), N, C, I,
+                                            _p(dx), _p(dg), _p(dwg), _p(dwu), _p(dwd))
+    return dx, dg, dwg, dwu, dwd

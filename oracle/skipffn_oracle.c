@@ -235,3 +235,97 @@ void skipffn_oracle_kept_cu_seqlens(const uint8_t *skip_mask, const int32_t *cu,
         kept_cu[s] = c;
     }
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Pre-norm variant.  The paper writes FFN(h_attn) (Eq. 4) and does not mention a normalisation,
+ * but the blocks of its LLaMA-3 / Vicuna backbones compute h + FFN(RMSNorm(h)).  This variant
+ * applies the textbook RMSNorm to the FFN input of retained tokens only:
+ *     rstd = 1 / sqrt(mean_c x[c]^2 + eps),   xn[c] = x[c] * rstd * gamma[c],
+ *     out  = x + FFN(xn)                      (skipped tokens: out = x, Eq. 5, unchanged).
+ * Backward is the exact derivative; with xh = x * rstd, gy = gamma * dxn:
+ *     dgamma[c] = sum over retained tokens of dxn[c] * xh[c]
+ *     dx[c]     = dout[c] + rstd * (gy[c] - xh[c] * mean_c(gy * xh)).
+ * Pins: rows of unit RMS with gamma = 1, eps = 0 reproduce the plain functions above exactly;
+ * scale invariance in x (eps = 0); fp64 autograd of a library restatement; finite differences.
+ */
+static double row_rstd(const double *xt, int64_t C, double eps)
+{
+    double ss = 0.0;
+    for (int64_t c = 0; c < C; ++c)
+        ss += xt[c] * xt[c];
+    return 1.0 / sqrt(ss / (double)C + eps);
+}
+
+void skipffn_oracle_forward_prenorm(const double *x, const uint8_t *skip_mask, const double *gamma,
+                                    double eps, const double *Wg, const double *Wu, const double *Wd,
+                                    int64_t N, int64_t C, int64_t I, double *out)
+{
+    double *xn = (double *)malloc(sizeof(double) * (size_t)C);
+    uint8_t keep = 0;
+    for (int64_t t = 0; t < N; ++t) {
+        const double *xt = x + t * C;
+        double *ot = out + t * C;
+        if (skip_mask[t] != 0) {
+            for (int64_t c = 0; c < C; ++c)
+                ot[c] = xt[c];
+            continue;
+        }
+        double rstd = row_rstd(xt, C, eps);
+        for (int64_t c = 0; c < C; ++c)
+            xn[c] = xt[c] * rstd * gamma[c];
+        /* FFN(xn) alone, then the residual of the un-normalised row */
+        skipffn_oracle_forward(xn, &keep, Wg, Wu, Wd, 1, C, I, 1, ot);
+        for (int64_t c = 0; c < C; ++c)
+            ot[c] += xt[c];
+    }
+    free(xn);
+}
+
+void skipffn_oracle_backward_prenorm(const double *x, const uint8_t *skip_mask, const double *gamma,
+                                     double eps, const double *Wg, const double *Wu, const double *Wd,
+                                     const double *dout, int64_t N, int64_t C, int64_t I, double *dx,
+                                     double *dgamma, double *dWg, double *dWu, double *dWd)
+{
+    double *xn = (double *)malloc(sizeof(double) * (size_t)C * 2);
+    double *dxn = xn + C;
+    double *tg = NULL, *tu = NULL, *td = NULL;
+    uint8_t keep = 0;
+    for (int64_t c = 0; c < C; ++c)
+        dgamma[c] = 0.0;
+    if (dWg) { memset(dWg, 0, sizeof(double) * (size_t)I * (size_t)C); tg = (double *)malloc(sizeof(double) * (size_t)I * (size_t)C); }
+    if (dWu) { memset(dWu, 0, sizeof(double) * (size_t)I * (size_t)C); tu = (double *)malloc(sizeof(double) * (size_t)I * (size_t)C); }
+    if (dWd) { memset(dWd, 0, sizeof(double) * (size_t)I * (size_t)C); td = (double *)malloc(sizeof(double) * (size_t)I * (size_t)C); }
+    for (int64_t t = 0; t < N; ++t) {
+        const double *xt = x + t * C, *dot = dout + t * C;
+        double *dxt = dx + t * C;
+        if (skip_mask[t] != 0) {
+            for (int64_t c = 0; c < C; ++c)
+                dxt[c] = dot[c];
+            continue;
+        }
+        double rstd = row_rstd(xt, C, eps);
+        for (int64_t c = 0; c < C; ++c)
+            xn[c] = xt[c] * rstd * gamma[c];
+        /* gradient of the FFN branch w.r.t. its input xn: the plain backward gives dout + that */
+        skipffn_oracle_backward(xn, &keep, Wg, Wu, Wd, dot, 1, C, I, dxn, tg, tu, td);
+        for (int64_t c = 0; c < C; ++c)
+            dxn[c] -= dot[c];
+        int64_t nW = I * C;
+        if (dWg) for (int64_t k = 0; k < nW; ++k) dWg[k] += tg[k];
+        if (dWu) for (int64_t k = 0; k < nW; ++k) dWu[k] += tu[k];
+        if (dWd) for (int64_t k = 0; k < nW; ++k) dWd[k] += td[k];
+        double m = 0.0;
+        for (int64_t c = 0; c < C; ++c) {
+            double xh = xt[c] * rstd;
+            dgamma[c] += dxn[c] * xh;
+            m += gamma[c] * dxn[c] * xh;
+        }
+        m /= (double)C;
+        for (int64_t c = 0; c < C; ++c) {
+            double xh = xt[c] * rstd;
+            dxt[c] = dot[c] + rstd * (gamma[c] * dxn[c] - xh * m);
+        }
+    }
+    free(xn);
+    free(tg); free(tu); free(td);
+}

@@ -318,3 +318,72 @@ def test_kv_compact_hand_cases_and_offsets():
     got = oracle.kept_cu_seqlens(w.skip_mask, w.cu_seqlens)
     want = [int((w.skip_mask[:c] == 0).sum()) for c in w.cu_seqlens]
     assert got.tolist() == want and got[-1] == w.n_kept
+
+
+# ------------------------------------------------------------------ pre-norm variant
+def test_prenorm_unit_rms_rows_reduce_to_plain_skipffn():
+    x, mask, wg, wu, wd, dout = _rand_case(11, 8, 12, seed=61)
+    x /= np.sqrt(np.mean(x * x, axis=1, keepdims=True))          # every row has RMS exactly 1
+    ones = np.ones(8)
+    a = oracle.forward_prenorm(x, mask, ones, 0.0, wg, wu, wd)
+    b = oracle.forward(x, mask, wg, wu, wd)
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-13)
+    # weight gradients see the same FFN input, so they agree too (dx does not: the norm has a Jacobian)
+    ga = oracle.backward_prenorm(x, mask, ones, 0.0, wg, wu, wd, dout)
+    gb = oracle.backward(x, mask, wg, wu, wd, dout)
+    for u, v in zip(ga[2:], gb[1:]):
+        np.testing.assert_allclose(u, v, rtol=1e-12, atol=1e-13)
+    sk = mask != 0
+    assert ga[0][sk].tobytes() == dout[sk].tobytes() and a[sk].tobytes() == x[sk].tobytes()
+
+
+def test_prenorm_closed_forms_and_scale_invariance():
+    # a constant row c: rstd = 1/|c| for eps = 0, so xn = sign(c) * gamma
+    C, I = 4, 3
+    r = np.random.default_rng(3)
+    wg, wu, wd = r.normal(size=(I, C)), r.normal(size=(I, C)), r.normal(size=(C, I))
+    gamma = r.normal(size=C)
+    x = np.full((1, C), -2.5)
+    out = oracle.forward_prenorm(x, [0], gamma, 0.0, wg, wu, wd)
+    want = x + oracle.forward(-gamma[None, :], [0], wg, wu, wd, ffn_only=True)
+    np.testing.assert_allclose(out, want, rtol=1e-13)
+    # eps: x = (3, 4, 0, 0), eps = 0.75 -> mean square 6.25, rstd = 1/sqrt(7) exactly as written
+    x = np.array([[3.0, 4.0, 0.0, 0.0]])
+    out = oracle.forward_prenorm(x, [0], gamma, 0.75, wg, wu, wd)
+    xn = x / math.sqrt(7.0) * gamma
+    np.testing.assert_allclose(out, x + oracle.forward(xn, [0], wg, wu, wd, ffn_only=True), rtol=1e-13)
+    # eps = 0: the FFN branch does not depend on the scale of x
+    x = r.normal(size=(5, C))
+    m = np.zeros(5, np.uint8)
+    a = oracle.forward_prenorm(x, m, gamma, 0.0, wg, wu, wd) - x
+    b = oracle.forward_prenorm(7.0 * x, m, gamma, 0.0, wg, wu, wd) - 7.0 * x
+    np.testing.assert_allclose(a, b, rtol=1e-11, atol=1e-12)
+
+
+def test_prenorm_backward_matches_fp64_autograd_and_finite_differences():
+    import torch
+    x, mask, wg, wu, wd, dout = _rand_case(9, 6, 10, seed=71)
+    gamma = np.random.default_rng(2).normal(size=6) + 1.0
+    eps = 1e-2
+    tx, tg, twg, twu, twd = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (x, gamma, wg, wu, wd))
+    keep = torch.tensor((mask == 0).astype(np.float64))[:, None]
+    xn = tx * torch.rsqrt((tx * tx).mean(dim=1, keepdim=True) + eps) * tg
+    out = tx + keep * ((torch.nn.functional.silu(xn @ twg.T) * (xn @ twu.T)) @ twd.T)
+    np.testing.assert_allclose(oracle.forward_prenorm(x, mask, gamma, eps, wg, wu, wd), out.detach().numpy(),
+                               rtol=1e-12, atol=1e-13)
+    (out * torch.tensor(dout)).sum().backward()
+    got = oracle.backward_prenorm(x, mask, gamma, eps, wg, wu, wd, dout)
+    for g, w in zip(got, (tx.grad, tg.grad, twg.grad, twu.grad, twd.grad)):
+        np.testing.assert_allclose(g, w.numpy(), rtol=1e-10, atol=1e-12)
+    # central differences on gamma and on one row of x
+    h = 1e-6
+    loss = lambda xx, gg: float(np.sum(dout * oracle.forward_prenorm(xx, mask, gg, eps, wg, wu, wd)))
+    for c in range(6):
+        gp, gm = gamma.copy(), gamma.copy()
+        gp[c] += h; gm[c] -= h
+        assert abs((loss(x, gp) - loss(x, gm)) / (2 * h) - got[1][c]) < 1e-6
+    t = int(np.flatnonzero(mask == 0)[0])
+    for c in range(6):
+        xp, xm = x.copy(), x.copy()
+        xp[t, c] += h; xm[t, c] -= h
+        assert abs((loss(xp, gamma) - loss(xm, gamma)) / (2 * h) - got[0][t, c]) < 1e-6
