@@ -175,6 +175,7 @@ def workload_config(args, w):
     return {"workload": f"{w.name} {args.shape}: C={w.C} I={w.I} N={w.N} tokens "
                         f"({w.meta.get('n_visual', '?')} visual + text per sequence), kept={w.n_kept}",
             "C": w.C, "I": w.I, "tokens": w.N, "kept_tokens": w.n_kept, "skip_ratio": args.skip_ratio,
+            "variant": "pre-norm (RMSNorm on the FFN input)" if args.prenorm else "as Eq. 4 (no normalisation)",
             "l2_policy": "inputs larger than L2 (weights 3 x %.0f MB re-read every step)" % (w.C * w.I * 2 / 1e6),
             "parallelism": "replicas only" if args.gpus > 1 else "single GPU"}
 
@@ -237,13 +238,18 @@ def run_ours(args):
     Wg, Wu, Wd = h_bf16(w.W_gate).to(dev), h_bf16(w.W_up).to(dev), h_bf16(w.W_down).to(dev)
     out, dx = torch.empty_like(x), torch.empty_like(x)
     dWg, dWu, dWd = torch.empty_like(Wg), torch.empty_like(Wu), torch.empty_like(Wd)
-    ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense)
+    ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense, prenorm=args.prenorm)
     if args.dense:
         nk = N
+    fwd_kw, bwd_kw = {}, {}
+    if args.prenorm:     # pre-norm variant: RMSNorm gain near 1, its gradient as one more output
+        gamma = h_bf16(1.0 + 0.1 * wl.normal(args.seed, 9, C)).to(dev)
+        fwd_kw = dict(gamma=gamma, eps=1e-5)
+        bwd_kw = dict(dgamma=torch.empty_like(gamma))
 
     def step():
-        ctx.forward(x, mask, Wg, Wu, Wd, out=out)
-        ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+        ctx.forward(x, mask, Wg, Wu, Wd, out=out, **fwd_kw)
+        ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd, **bwd_kw)
 
     # End-to-end leg: every step copies x, skip_mask and dout from pinned host memory and copies
     # out and dx back.  Two sets of device buffers and three streams (host->device, compute,
@@ -271,8 +277,8 @@ def run_ours(args):
         s_comp.wait_event(b["ready_in"])
         if not first_use:
             s_comp.wait_event(b["copied_out"])      # its previous results are on the host
-        ctx.forward(b["x"], b["mask"], Wg, Wu, Wd, out=b["out"])
-        ctx.backward(b["dout"], dx=b["dx"], dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+        ctx.forward(b["x"], b["mask"], Wg, Wu, Wd, out=b["out"], **fwd_kw)
+        ctx.backward(b["dout"], dx=b["dx"], dW_gate=dWg, dW_up=dWu, dW_down=dWd, **bwd_kw)
         b["done"].record(s_comp)
         with torch.cuda.stream(s_out):
             s_out.wait_event(b["done"])
@@ -555,6 +561,8 @@ def main():
     ap.add_argument("--shape", default="llama3-8b", choices=list(wl.SWEEP_SHAPES))
     ap.add_argument("--skip-ratio", type=float, default=0.75)
     ap.add_argument("--dense", action="store_true", help="in-library dense comparator (mask ignored)")
+    ap.add_argument("--prenorm", action="store_true",
+                    help="pre-norm variant: out = x + FFN(RMSNorm(x) * gamma), with dgamma in the backward")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -56,7 +56,7 @@ typedef struct {
     int32_t grad_dtype_fp32; /* 1: dW_* are fp32 regardless of dtype */
     int32_t accumulate_dw;   /* 1: dW += ..., 0: dW is overwritten */
     int32_t path;            /* skipffn_path */
-    int32_t reserved;        /* must be 0 */
+    int32_t prenorm;         /* 1: pre-norm variant (skipffn_forward_prenorm / _backward_prenorm) */
 } skipffn_config;
 
 /* Host-side handle linking one forward call to its backward call.  It points into the caller's
@@ -98,6 +98,24 @@ skipffn_status skipffn_forward(skipffn_saved *saved, const void *x, const uint8_
 skipffn_status skipffn_backward(const void *dout, skipffn_saved *saved, void *dx, void *dW_gate,
                                 void *dW_up, void *dW_down, void *stream);
 
+/* Pre-norm variant (cfg.prenorm = 1).  Eq. 4 writes FFN(h_attn); the decoder blocks of the paper's
+ * LLaMA-3 / Vicuna backbones (section 6.4 training setup) normalise the FFN input, so this variant
+ * computes, for retained tokens,
+ *     out[t] = x[t] + FFN( RMSNorm(x[t]) * gamma ),   RMSNorm(x) = x / sqrt(mean_c x[c]^2 + eps),
+ * and out[t] = x[t] for skipped tokens (Eq. 5): skipping the FFN skips its normalisation too.
+ * gamma: [C] in cfg.dtype (borrowed until the backward returns); eps >= 0.  The normalised rows
+ * are rounded once to cfg.dtype before the projections; statistics are fp32.
+ * Backward additionally returns dgamma [C] (cfg.dtype, fp32 with grad_dtype_fp32; overwritten or
+ * accumulated like the weight gradients; may be NULL).  All other arguments as in
+ * skipffn_forward / skipffn_backward, which reject a handle created with prenorm = 1 (and these
+ * two reject one created without). */
+skipffn_status skipffn_forward_prenorm(skipffn_saved *saved, const void *x, const uint8_t *skip_mask,
+                                       int64_t B, int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
+                                       const void *gamma, float eps, const void *W_gate,
+                                       const void *W_up, const void *W_down, void *out, void *stream);
+skipffn_status skipffn_backward_prenorm(const void *dout, skipffn_saved *saved, void *dx, void *dgamma,
+                                        void *dW_gate, void *dW_up, void *dW_down, void *stream);
+
 /* Device addresses of the kept-row index list (int32, ascending) and of its length. */
 skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
                                 const int32_t **nk_dev);
@@ -121,7 +139,8 @@ skipffn_status skipffn_kv_compact(const skipffn_saved *saved, const void *src, v
 
 /* Device addresses of the compacted intermediates of the last forward / backward, each
  * [round_up(Nk,128), I] in cfg.dtype (rows >= Nk are zero): which = 0 G, 1 U, 2 H, 3 dG, 4 dU;
- * 5 = kept rows of x [.., C]; 6 = kept rows of dout [.., C]. */
+ * 5 = kept rows of x [.., C]; 6 = kept rows of dout [.., C]; 7 = normalised kept rows of x
+ * [.., C] (pre-norm variant only). */
 skipffn_status skipffn_get_intermediate(const skipffn_saved *saved, int32_t which,
                                         const void **ptr_dev);
 
@@ -137,8 +156,8 @@ skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_ou
  * 2 gate/up GEMM, 3 down GEMM, 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate, 8 dW_up,
  * 9 dX GEMM.  The tensor-core path computes the requested weight gradients in ONE grouped launch,
  * whose time is reported in the slot of the first of them (6 when dW_down is requested) with the
- * other two slots 0. */
-#define SKIPFFN_PROFILE_SLOTS 10
+ * other two slots 0.  Slot 10 (pre-norm variant): the normalisation's backward (dx rows and dgamma). */
+#define SKIPFFN_PROFILE_SLOTS 11
 skipffn_status skipffn_profile_enable(skipffn_saved *saved, int32_t on);
 skipffn_status skipffn_profile_read(skipffn_saved *saved, float *ms);
 

@@ -17,11 +17,12 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_plan", "skipffn_forward", "skipffn_backward", "skipffn_get_kept",
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
            "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
-           "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact"]
+           "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact",
+           "skipffn_forward_prenorm", "skipffn_backward_prenorm"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
-                 "dw_up", "dx"]
+                 "dw_up", "dx", "norm_bwd"]
 
 
 class SkipFFNError(RuntimeError):
@@ -34,7 +35,7 @@ class _Config(ctypes.Structure):
     _fields_ = [("C", ctypes.c_int32), ("I", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("dense", ctypes.c_int32), ("grad_dtype_fp32", ctypes.c_int32),
                 ("accumulate_dw", ctypes.c_int32), ("path", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("prenorm", ctypes.c_int32)]
 
 
 def load_library() -> ctypes.CDLL:
@@ -60,6 +61,10 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_forward.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, vp]
     lib.skipffn_backward.restype = i32
     lib.skipffn_backward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.skipffn_forward_prenorm.restype = i32
+    lib.skipffn_forward_prenorm.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.skipffn_backward_prenorm.restype = i32
+    lib.skipffn_backward_prenorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.skipffn_get_kept.restype = i32
     lib.skipffn_get_kept.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.skipffn_get_intermediate.restype = i32
@@ -86,9 +91,10 @@ def load_library() -> ctypes.CDLL:
     return lib
 
 
-def _cfg(C, I, dtype=BF16, dense=False, grad_fp32=False, accumulate_dw=False, path=PATH_DEFAULT):
+def _cfg(C, I, dtype=BF16, dense=False, grad_fp32=False, accumulate_dw=False, path=PATH_DEFAULT,
+         prenorm=False):
     return _Config(int(C), int(I), int(dtype), int(bool(dense)), int(bool(grad_fp32)),
-                   int(bool(accumulate_dw)), int(path), 0)
+                   int(bool(accumulate_dw)), int(path), int(bool(prenorm)))
 
 
 def skipffn_workspace_bytes(C, I, max_tokens, dtype=BF16) -> int:
@@ -159,7 +165,7 @@ class SkipFFN:
 
     def __init__(self, C: int, I: int, max_tokens: int, dtype: int = BF16, dense: bool = False,
                  grad_fp32: bool = False, accumulate_dw: bool = False, path: int = PATH_DEFAULT,
-                 device="cuda"):
+                 device="cuda", prenorm: bool = False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("Skip-FFN needs a CUDA device (sm_100a); there is no CPU path")
@@ -167,7 +173,8 @@ class SkipFFN:
         self.lib = load_library()
         self.C, self.I, self.dtype, self.max_tokens = int(C), int(I), int(dtype), int(max_tokens)
         self.grad_fp32 = bool(grad_fp32) or dtype == FP32
-        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path)
+        self.prenorm = bool(prenorm)
+        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path, prenorm)
         self.device = torch.device(device)
         nbytes = int(self.lib.skipffn_workspace_bytes(ctypes.byref(self.cfg), self.max_tokens))
         if nbytes == 0:
@@ -213,8 +220,11 @@ class SkipFFN:
         if st != 0:
             raise SkipFFNError(st, "skipffn_plan")
 
-    def forward(self, x, skip_mask, W_gate, W_up, W_down, out=None, cu_seqlens=None):
-        """x: [B, S, C] or [N, C]; skip_mask: uint8 [B, S] / [N] or None (reuse the planned list)."""
+    def forward(self, x, skip_mask, W_gate, W_up, W_down, out=None, cu_seqlens=None, gamma=None,
+                eps: float = 1e-5):
+        """x: [B, S, C] or [N, C]; skip_mask: uint8 [B, S] / [N] or None (reuse the planned list).
+        A context created with ``prenorm=True`` takes the gain vector ``gamma`` [C] and ``eps`` and
+        calls ``skipffn_forward_prenorm``."""
         torch, dt = self._torch, self.torch_dtype
         if x.dim() == 2:
             B, S = 1, x.shape[0]
@@ -238,17 +248,29 @@ class SkipFFN:
             vals = [int(v) for v in cu_seqlens]
             n_seq = len(vals) - 1
             cu_arr = (ctypes.c_int32 * len(vals))(*vals)
-        st = self.lib.skipffn_forward(self._saved, _ptr(x), _ptr(skip_mask), B, S,
-                                      ctypes.cast(cu_arr, ctypes.c_void_p) if cu_arr is not None else None,
-                                      n_seq, _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(out),
-                                      self._stream())
+        cu_p = ctypes.cast(cu_arr, ctypes.c_void_p) if cu_arr is not None else None
+        if self.prenorm:
+            self._check(gamma, "gamma", (self.C,), dt)
+            if gamma is None:
+                raise ValueError("a pre-norm context needs gamma")
+            st = self.lib.skipffn_forward_prenorm(self._saved, _ptr(x), _ptr(skip_mask), B, S, cu_p, n_seq,
+                                                  _ptr(gamma), ctypes.c_float(eps), _ptr(W_gate), _ptr(W_up),
+                                                  _ptr(W_down), _ptr(out), self._stream())
+        else:
+            if gamma is not None:
+                raise ValueError("gamma needs a context created with prenorm=True")
+            st = self.lib.skipffn_forward(self._saved, _ptr(x), _ptr(skip_mask), B, S, cu_p,
+                                          n_seq, _ptr(W_gate), _ptr(W_up), _ptr(W_down), _ptr(out),
+                                          self._stream())
         if st != 0:
             raise SkipFFNError(st, "skipffn_forward")
-        self._keep = [W_gate, W_up, W_down]
+        self._keep = [W_gate, W_up, W_down, gamma]
         self._shape = tuple(x.shape)
         return out
 
-    def backward(self, dout, dx=None, dW_gate=None, dW_up=None, dW_down=None, need_dw=True):
+    def backward(self, dout, dx=None, dW_gate=None, dW_up=None, dW_down=None, need_dw=True, dgamma=None):
+        """Returns ``(dx, dW_gate, dW_up, dW_down)``; a pre-norm context returns
+        ``(dx, dW_gate, dW_up, dW_down, dgamma)``."""
         torch, dt = self._torch, self.torch_dtype
         if self._shape is None:
             raise SkipFFNError(1, "skipffn_backward (no forward has run on this context)")
@@ -267,6 +289,15 @@ class SkipFFN:
         self._check(dW_gate, "dW_gate", (self.I, self.C), gdt)
         self._check(dW_up, "dW_up", (self.I, self.C), gdt)
         self._check(dW_down, "dW_down", (self.C, self.I), gdt)
+        if self.prenorm:
+            if dgamma is None and need_dw:
+                dgamma = torch.empty(self.C, dtype=gdt, device=self.device)
+            self._check(dgamma, "dgamma", (self.C,), gdt)
+            st = self.lib.skipffn_backward_prenorm(_ptr(dout), self._saved, _ptr(dx), _ptr(dgamma), _ptr(dW_gate),
+                                                   _ptr(dW_up), _ptr(dW_down), self._stream())
+            if st != 0:
+                raise SkipFFNError(st, "skipffn_backward_prenorm")
+            return dx, dW_gate, dW_up, dW_down, dgamma
         st = self.lib.skipffn_backward(_ptr(dout), self._saved, _ptr(dx), _ptr(dW_gate),
                                        _ptr(dW_up), _ptr(dW_down), self._stream())
         if st != 0:
@@ -331,7 +362,7 @@ class SkipFFN:
         st = self.lib.skipffn_get_intermediate(self._saved, which, ctypes.byref(p))
         if st != 0:
             raise SkipFFNError(st, "skipffn_get_intermediate")
-        cols = self.I if which < 5 else self.C
+        cols = self.I if which < 5 else self.C   # 5 Xk, 6 dOk, 7 normalised Xk
         return self._view(p.value, rows * cols, self.torch_dtype).view(rows, cols).clone()
 
     def _view(self, ptr, numel, dtype):

@@ -15,6 +15,10 @@ struct skipffn_saved {
     // workspace carve-up (device)
     int32_t *status, *sk_flags, *idx, *pos;
     void *sk_slots, *Xk, *dOk, *G, *U, *H, *dG, *dU;
+    void *Xn;              // pre-norm variant: normalised kept rows (the FFN input)
+    float *rstd, *dY;      //   per-row 1/rms, and the fp32 gradient w.r.t. the normalised rows
+    float *dg_part;        //   [DG_CHUNKS, C] partial sums of the gain's gradient
+    const void *gamma;     //   gain vector of the last forward (borrowed)
     // state
     int64_t planned_N;     // tokens of the current index list, -1 if none
     int forwarded;
@@ -30,13 +34,14 @@ struct skipffn_saved {
 namespace {
 
 struct Layout {
-    size_t status, idx, pos, sk_slots, Xk, dOk, G, U, H, dG, dU, total;
+    size_t status, idx, pos, sk_slots, Xk, dOk, G, U, H, dG, dU, Xn, rstd, dY, dg_part, total;
 };
 
 bool valid_cfg(const skipffn_config *c)
 {
     return c && c->C > 0 && c->I > 0 && (c->dtype == SKIPFFN_BF16 || c->dtype == SKIPFFN_FP32) &&
-           (c->path == SKIPFFN_PATH_DEFAULT || c->path == SKIPFFN_PATH_SIMT) && c->reserved == 0;
+           (c->path == SKIPFFN_PATH_DEFAULT || c->path == SKIPFFN_PATH_SIMT) &&
+           (c->prenorm == 0 || c->prenorm == 1);
 }
 
 Layout make_layout(const skipffn_config *c, int64_t max_tokens)
@@ -57,6 +62,10 @@ Layout make_layout(const skipffn_config *c, int64_t max_tokens)
     l.H = take((size_t)cap * c->I * es);
     l.dG = take((size_t)cap * c->I * es);
     l.dU = take((size_t)cap * c->I * es);
+    l.Xn = take(c->prenorm ? (size_t)cap * c->C * es : 0);
+    l.rstd = take(c->prenorm ? (size_t)cap * 4 : 0);
+    l.dY = take(c->prenorm ? (size_t)cap * c->C * 4 : 0);
+    l.dg_part = take(c->prenorm ? (size_t)DG_CHUNKS * c->C * 4 : 0);
     l.total = off;
     return l;
 }
@@ -72,7 +81,7 @@ bool use_umma(const skipffn_saved *s)
 // 2 gate/up GEMM, 3 down GEMM; backward 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate,
 // 8 dW_up, 9 dX GEMM.
 enum : int { SLOT_COMPACT = 0, SLOT_ROUTE_X, SLOT_GATEUP, SLOT_DOWN, SLOT_ROUTE_DOUT, SLOT_DH,
-             SLOT_DW_DOWN, SLOT_DW_GATE, SLOT_DW_UP, SLOT_DX };
+             SLOT_DW_DOWN, SLOT_DW_GATE, SLOT_DW_UP, SLOT_DX, SLOT_NORM_BWD };
 
 template <typename F>
 cudaError_t timed_launch(skipffn_saved *s, int slot, cudaStream_t st, F &&launch)
@@ -160,6 +169,8 @@ skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config 
     s->pos = (int32_t *)(w + l.pos);
     s->Xk = w + l.Xk; s->dOk = w + l.dOk;
     s->G = w + l.G; s->U = w + l.U; s->H = w + l.H; s->dG = w + l.dG; s->dU = w + l.dU;
+    s->Xn = w + l.Xn; s->rstd = (float *)(w + l.rstd); s->dY = (float *)(w + l.dY);
+    s->dg_part = (float *)(w + l.dg_part);
     s->planned_N = -1;
     *saved = s;
     return SKIPFFN_OK;
@@ -217,12 +228,14 @@ skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t 
     return do_plan(s, skip_mask, N, 0, st);
 }
 
-skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
-                               int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
-                               const void *W_gate, const void *W_up, const void *W_down, void *out,
-                               void *stream)
+static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
+                                   int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
+                                   const void *gamma, float eps, const void *W_gate, const void *W_up,
+                                   const void *W_down, void *out, void *stream)
 {
     if (!s || B < 0 || S < 0) return SKIPFFN_EINVAL;
+    if ((s->cfg.prenorm != 0) != (gamma != nullptr)) return SKIPFFN_EINVAL;   // wrong entry point
+    if (gamma && (!aligned16(gamma) || !(eps >= 0.0f))) return SKIPFFN_EINVAL;
     const int64_t N = B * S;
     if (N > s->max_tokens) return SKIPFFN_EINVAL;
     if (!W_gate || !W_up || !W_down || (N > 0 && (!x || !out))) return SKIPFFN_EINVAL;
@@ -246,19 +259,21 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
         if (s->planned_N != N) return SKIPFFN_EINVAL;   // no list to reuse
         s->launches[0] = 0;
     }
-    s->Wg = W_gate; s->Wu = W_up; s->Wd = W_down;
+    s->Wg = W_gate; s->Wu = W_up; s->Wd = W_down; s->gamma = gamma;
     if (N == 0) { s->forwarded = 1; return SKIPFFN_OK; }
 
     // kept rows of x -> Xk (also the residual stash when out aliases x); skipped rows -> out
     RouteArgs r;
     r.src = x; r.dst_compact = s->Xk; r.dst_identity = out; r.pos = s->pos; r.status = s->status;
     r.N = N; r.C = C; r.elem_bytes = s->esize;
-    if (timed_launch(s, SLOT_ROUTE_X, st, [&] { return launch_route(r, st); }) != cudaSuccess)
+    if (timed_launch(s, SLOT_ROUTE_X, st, [&] {
+            return gamma ? launch_route_norm(r, s->Xn, s->rstd, gamma, eps, st) : launch_route(r, st);
+        }) != cudaSuccess)
         return SKIPFFN_ECUDA;
 
-    // G = Xk Wg^T, U = Xk Wu^T, H = silu(G) * U
+    // G = A Wg^T, U = A Wu^T, H = silu(G) * U, with A = the kept rows (normalised in the pre-norm variant)
     GemmArgs g = base_args(s);
-    g.A = s->Xk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+    g.A = gamma ? s->Xn : s->Xk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
     g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
     g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
     g.out0 = s->G; g.out1 = s->U; g.out2 = s->H; g.ldo = I;
@@ -275,10 +290,30 @@ skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *s
     return SKIPFFN_OK;
 }
 
-skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, void *dW_gate,
-                                void *dW_up, void *dW_down, void *stream)
+skipffn_status skipffn_forward(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
+                               int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
+                               const void *W_gate, const void *W_up, const void *W_down, void *out,
+                               void *stream)
+{
+    return forward_impl(s, x, skip_mask, B, S, cu_seqlens, n_seq, nullptr, 0.0f, W_gate, W_up, W_down, out, stream);
+}
+
+skipffn_status skipffn_forward_prenorm(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
+                                       int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
+                                       const void *gamma, float eps, const void *W_gate, const void *W_up,
+                                       const void *W_down, void *out, void *stream)
+{
+    if (!gamma) return SKIPFFN_EINVAL;
+    return forward_impl(s, x, skip_mask, B, S, cu_seqlens, n_seq, gamma, eps, W_gate, W_up, W_down, out, stream);
+}
+
+static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx, void *dgamma, void *dW_gate,
+                                    void *dW_up, void *dW_down, void *stream)
 {
     if (!s || !s->forwarded) return SKIPFFN_EINVAL;
+    const bool prenorm = s->cfg.prenorm != 0;
+    if (!prenorm && dgamma) return SKIPFFN_EINVAL;
+    if (!aligned16(dgamma)) return SKIPFFN_EINVAL;
     const int64_t N = s->planned_N;
     if (N > 0 && (!dout || !dx)) return SKIPFFN_EINVAL;
     if (!aligned16(dout) || !aligned16(dx) || !aligned16(dW_gate) || !aligned16(dW_up) || !aligned16(dW_down))
@@ -319,7 +354,8 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         if (w == 0) {
             q.A = s->dOk; q.lda_k = C; q.B = s->H; q.ldb_k = I; q.M = C; q.N = I; q.ldo = I;
         } else {
-            q.A = w == 1 ? s->dG : s->dU; q.lda_k = I; q.B = s->Xk; q.ldb_k = C; q.M = I; q.N = C; q.ldo = C;
+            q.A = w == 1 ? s->dG : s->dU; q.lda_k = I; q.B = prenorm ? s->Xn : s->Xk; q.ldb_k = C;
+            q.M = I; q.N = C; q.ldo = C;
         }
         q.lda_m = 1; q.ldb_n = 1; q.a_outer = s->cap; q.b_outer = s->cap;
         q.K = kmax; q.k_from_nk = 1;
@@ -344,10 +380,39 @@ skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, vo
         g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
         g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
         g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
-        g.in0 = s->dOk; g.out0 = dx; g.ldo = C;
+        if (prenorm) { g.in0 = nullptr; g.out0 = s->dY; g.out_fp32 = 1; }   // gradient w.r.t. the normalised rows
+        else { g.in0 = s->dOk; g.out0 = dx; }
+        g.ldo = C;
         if (run_gemm(s, SLOT_DX, EPI_DX, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     }
+    if (prenorm) {   // through the normalisation: dx rows (scattered) and the gain's gradient
+        const int gfp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
+        if (N == 0 && dgamma && !s->cfg.accumulate_dw) {
+            if (cudaMemsetAsync(dgamma, 0, (size_t)C * (gfp32 ? 4 : 2), st) != cudaSuccess) return SKIPFFN_ECUDA;
+        } else if (N > 0) {
+            if (timed_launch(s, SLOT_NORM_BWD, st, [&] {
+                    return launch_norm_bwd(s->dY, s->Xk, s->dOk, s->rstd, s->gamma, dx, dgamma, s->dg_part, s->idx, s->status,
+                                           N, C, s->esize, gfp32, s->cfg.accumulate_dw, st);
+                }) != cudaSuccess)
+                return SKIPFFN_ECUDA;
+            if (dgamma) s->launches[1] += 2;   // the slot covers three kernels: rows, then the gain's gradient in two stages
+        }
+    }
     return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_backward(const void *dout, skipffn_saved *s, void *dx, void *dW_gate,
+                                void *dW_up, void *dW_down, void *stream)
+{
+    if (s && s->cfg.prenorm) return SKIPFFN_EINVAL;   // wrong entry point
+    return backward_impl(dout, s, dx, nullptr, dW_gate, dW_up, dW_down, stream);
+}
+
+skipffn_status skipffn_backward_prenorm(const void *dout, skipffn_saved *s, void *dx, void *dgamma,
+                                        void *dW_gate, void *dW_up, void *dW_down, void *stream)
+{
+    if (s && !s->cfg.prenorm) return SKIPFFN_EINVAL;
+    return backward_impl(dout, s, dx, dgamma, dW_gate, dW_up, dW_down, stream);
 }
 
 skipffn_status skipffn_kv_compact(const skipffn_saved *s, const void *src, void *dst, int64_t planes,
@@ -386,8 +451,8 @@ skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev,
 skipffn_status skipffn_get_intermediate(const skipffn_saved *s, int32_t which, const void **ptr_dev)
 {
     if (!s || !ptr_dev) return SKIPFFN_EINVAL;
-    const void *t[7] = {s->G, s->U, s->H, s->dG, s->dU, s->Xk, s->dOk};
-    if (which < 0 || which > 6) return SKIPFFN_EINVAL;
+    const void *t[8] = {s->G, s->U, s->H, s->dG, s->dU, s->Xk, s->dOk, s->Xn};
+    if (which < 0 || which > 7 || (which == 7 && !s->cfg.prenorm)) return SKIPFFN_EINVAL;
     *ptr_dev = t[which];
     return SKIPFFN_OK;
 }

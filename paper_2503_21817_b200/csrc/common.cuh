@@ -94,6 +94,14 @@ cudaError_t launch_kv_compact(const void *src, void *dst, const int32_t *idx, co
                               cudaStream_t s);
 cudaError_t launch_kept_cu_seqlens(const int32_t *cu, int32_t *new_cu, int n, const int32_t *idx,
                                    const int32_t *status, cudaStream_t s);
+// prenorm.cu
+cudaError_t launch_route_norm(const RouteArgs &a, void *Xn, float *rstd, const void *gamma, float eps,
+                              cudaStream_t s);
+cudaError_t launch_norm_bwd(const float *dY, const void *Xk, const void *dOk, const float *rstd,
+                            const void *gamma, void *dx, void *dgamma, float *dg_part, const int32_t *idx,
+                            const int32_t *status, int64_t max_rows, int C, int elem_bytes,
+                            int dgamma_fp32, int accumulate, cudaStream_t s);
+constexpr int DG_CHUNKS = 32;   // row chunks of the two-stage dgamma reduction ([DG_CHUNKS, C] fp32 partials)
 // simt.cu
 cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
 // umma.cu (bf16 only)

@@ -91,6 +91,8 @@ __global__ void __launch_bounds__(ST_THREADS) k_simt_gemm(GemmArgs a)
                 ((T *)a.out0)[o] = from_f32<T>(v);
                 ((T *)a.out1)[o] = from_f32<T>(u);
                 ((T *)a.out2)[o] = from_f32<T>(swiglu(v, u));   // from the fp32 accumulators
+            } else if (EPI == EPI_DX && a.out_fp32) {        // pre-norm variant: raw fp32 rows, compact
+                ((float *)a.out0)[o] = v;
             } else if (EPI == EPI_DOWN || EPI == EPI_DX) {   // residual add + row scatter
                 float res = to_f32(((const T *)a.in0)[o]);   // compacted residual row
                 int64_t tok = a.idx[m];

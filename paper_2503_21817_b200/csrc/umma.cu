@@ -687,7 +687,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             // prefetch of the per-row epilogue inputs of the first chunk (overlaps the accumulator wait)
             uint4 pa[4], pb[4];
             auto prefetch = [&](int n) {
-                if (EPI == EPI_DH || EPI == EPI_DOWN || EPI == EPI_DX) {
+                if ((EPI == EPI_DH || EPI == EPI_DOWN || EPI == EPI_DX) && p.in0 != nullptr) {
                     const int64_t o = (int64_t)m * p.ldo + n;
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
@@ -783,6 +783,17 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         w[q] = pack_bf16(fast_swiglu(__uint_as_float(r[2 * q]), __uint_as_float(r2[GATEUP ? 2 * q : 0])),
                                          fast_swiglu(__uint_as_float(r[2 * q + 1]), __uint_as_float(r2[GATEUP ? 2 * q + 1 : 0])));
                     store_rows_64B(sbuf, lane, w, rowH, valid_slots);
+                } else if (EPI == EPI_DX && p.out_fp32) {
+                    // pre-norm variant: the raw fp32 gradient w.r.t. the normalised rows, compact,
+                    // no residual (the normalisation's backward runs afterwards, row-wide)
+                    char *row = row_valid ? (char *)p.out0 + ((int64_t)m * p.ldo + n) * 4 : nullptr;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) w[q] = r[hh * 16 + q];
+                        store_rows_64B_f32(sbuf, lane, w, row ? row + hh * 64 : nullptr,
+                                           min(4, max(0, (n_end - n - hh * 16) / 4)), 0);
+                    }
                 } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
                     // residual add in fp32, one rounding, scatter to the token's row
                     const uint32_t rw[16] = {ca[0].x, ca[0].y, ca[0].z, ca[0].w, ca[1].x, ca[1].y, ca[1].z, ca[1].w,
