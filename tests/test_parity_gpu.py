@@ -316,3 +316,36 @@ def test_config3_highres_full_size_sampled():
     w = wl.config3()
     assert (w.N, w.n_kept) == (9376, 1312)
     _sampled_full_size(w, n_tok=6, n_col=4)
+
+
+def test_config4_packed_full_size_sampled():
+    # 16 packed sequences, about 32 k tokens of which about 11 k are kept
+    w = wl.config4()
+    assert w.cu_seqlens.shape == (17,) and 25000 < w.N < 40000 and w.n_kept > 8000
+    _sampled_full_size(w, n_tok=6, n_col=3)
+
+
+@pytest.mark.parametrize("ratio", [0.0, 1.0])
+def test_sweep_end_points_vicuna_13b_shape_sampled(ratio):
+    # the other shape of the skip-ratio sweep (C = 5120, I = 13824) at its two extremes: every
+    # visual token kept (4928 rows) and every visual token skipped (320 text rows)
+    C, I = wl.SWEEP_SHAPES["vicuna-13b"]
+    w = wl.config2(skip_ratio=ratio, C=C, I=I)
+    assert w.n_kept == (4928 if ratio == 0.0 else 320)
+    r = _sampled_full_size(w, n_tok=5, n_col=3) if ratio else None
+    if ratio == 0.0:
+        # no skipped token to sample: same checks without the skipped rows
+        r = run(w)
+        rng = np.random.default_rng(0)
+        tok = rng.choice(w.N, 6, replace=False).astype(np.int64)
+        cols = rng.choice(w.I, 3, replace=False).astype(np.int64)
+        x64, wg, wu, wd, do = (a.astype(np.float64) for a in (w.x, w.W_gate, w.W_up, w.W_down, w.dout))
+        out_r, dx_r = oracle.rows(x64, w.skip_mask, wg, wu, wd, do, tok)
+        check(to_host(r["out"].reshape(w.N, w.C)[tok]), out_r, "bf16", "out rows")
+        check(to_host(r["dx"].reshape(w.N, w.C)[tok]), dx_r, "bf16", "dx rows")
+        a, b, c = oracle.dw_columns(x64, w.skip_mask, wg, wu, wd, do, cols)
+        check(to_host(r["dW_gate"][cols]), a, "bf16", "dW_gate rows")
+        check(to_host(r["dW_up"][cols]), b, "bf16", "dW_up rows")
+        check(to_host(r["dW_down"][:, cols].T), c, "bf16", "dW_down cols")
+        idx, nk = r["ctx"].kept()
+        assert nk == w.N and np.array_equal(idx.cpu().numpy(), np.arange(w.N))
