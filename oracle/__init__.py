@@ -53,6 +53,10 @@ def _load() -> ctypes.CDLL:
         lib.skipffn_oracle_backward_prenorm.restype = None
         lib.skipffn_oracle_backward_prenorm.argtypes = [dp, bp, dp, ctypes.c_double, dp, dp, dp, dp, i64, i64, i64,
                                                         dp, dp, dp, dp, dp]
+        lib.skipffn_oracle_summary_forward.restype = None
+        lib.skipffn_oracle_summary_forward.argtypes = [dp, ctypes.c_void_p, i64, i64, dp, dp, dp]
+        lib.skipffn_oracle_summary_backward.restype = None
+        lib.skipffn_oracle_summary_backward.argtypes = [dp, ctypes.c_void_p, i64, i64, dp, dp, dp, dp]
         lib.skipffn_oracle_kv_compact.restype = i64
         lib.skipffn_oracle_kv_compact.argtypes = [bp, bp, i64, i64, i64, bp]
         lib.skipffn_oracle_kept_cu_seqlens.restype = None
@@ -197,3 +201,27 @@ def backward_prenorm(x, skip_mask, gamma, eps, W_gate, W_up, W_down, dout, need_
     _load().skipffn_oracle_backward_prenorm(_p(x), _p(m), _p(g), float(eps), _p(wg), _p(wu), _p(wd), _p(do), N, C, I,
                                             _p(dx), _p(dg), _p(dwg), _p(dwu), _p(dwd))
     return dx, dg, dwg, dwu, dwd
+
+
+def summary_forward(X, offsets, w):
+    """Adaptive summary tokens (Eq. 6): ``(xs [n_seg, C], probs [n])`` for packed ``X [n, C]`` whose
+    segment s is rows ``offsets[s] .. offsets[s+1]-1``."""
+    X, w = _f64(X), _f64(w)
+    off = np.ascontiguousarray(offsets, dtype=np.int32)
+    n, C = X.shape
+    assert w.shape == (C,) and off[0] == 0 and off[-1] == n and np.all(np.diff(off) >= 0)
+    xs = np.empty((off.size - 1, C), dtype=np.float64)
+    probs = np.zeros(max(n, 1), dtype=np.float64)
+    _load().skipffn_oracle_summary_forward(_p(X), _p(off), off.size - 1, C, _p(w), _p(xs), _p(probs))
+    return xs, probs[:n]
+
+
+def summary_backward(X, offsets, w, dxs):
+    """``(dX [n, C], dw [C])`` of the adaptive summary layer for the loss ``sum(dxs * xs)``."""
+    X, w, dxs = _f64(X), _f64(w), _f64(dxs)
+    off = np.ascontiguousarray(offsets, dtype=np.int32)
+    n, C = X.shape
+    dX = np.zeros((n, C), dtype=np.float64)
+    dw = np.empty(C, dtype=np.float64)
+    _load().skipffn_oracle_summary_backward(_p(X), _p(off), off.size - 1, C, _p(w), _p(dxs), _p(dX), _p(dw))
+    return dX, dw

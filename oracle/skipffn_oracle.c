@@ -329,3 +329,77 @@ void skipffn_oracle_backward_prenorm(const double *x, const uint8_t *skip_mask, 
     free(xn);
     free(tg); free(tu); free(td);
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Adaptive summary token (section 4.2, Eq. 6):  x_s = softmax(X w^T)^T X, with X [n, C] the retained
+ * or skipped visual tokens of one sample and w [C] the layer's only weight.  Segments of a packed
+ * X are processed independently: rows off[s] .. off[s+1]-1 give xs[s].  An empty segment gives 0.
+ * Backward for L = sum(dxs * xs): with p = softmax(X w), a_i = dxs . X_i, t = sum_j p_j a_j,
+ * ds_i = p_i (a_i - t):   dX_i = p_i dxs + ds_i w,   dw = sum_i ds_i X_i.
+ * Pins: w = 0 gives the mean of the rows; a one-row segment returns the row; a large score gap
+ * selects one row; the softmax weights are a library softmax; fp64 autograd; finite differences.
+ */
+void skipffn_oracle_summary_forward(const double *X, const int32_t *off, int64_t n_seg, int64_t C,
+                                    const double *w, double *xs, double *probs)
+{
+    for (int64_t s = 0; s < n_seg; ++s) {
+        int64_t lo = off[s], hi = off[s + 1];
+        double *y = xs + s * C;
+        for (int64_t c = 0; c < C; ++c)
+            y[c] = 0.0;
+        if (hi <= lo)
+            continue;
+        double mx = -INFINITY;
+        for (int64_t i = lo; i < hi; ++i) {
+            double sc = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                sc += X[i * C + c] * w[c];
+            probs[i] = sc;
+            if (sc > mx)
+                mx = sc;
+        }
+        double den = 0.0;
+        for (int64_t i = lo; i < hi; ++i) {
+            probs[i] = exp(probs[i] - mx);
+            den += probs[i];
+        }
+        for (int64_t i = lo; i < hi; ++i) {
+            probs[i] /= den;
+            for (int64_t c = 0; c < C; ++c)
+                y[c] += probs[i] * X[i * C + c];
+        }
+    }
+}
+
+void skipffn_oracle_summary_backward(const double *X, const int32_t *off, int64_t n_seg, int64_t C,
+                                     const double *w, const double *dxs, double *dX, double *dw)
+{
+    int64_t total = off[n_seg];
+    double *probs = (double *)malloc(sizeof(double) * (size_t)(total > 0 ? total : 1));
+    double *xs = (double *)malloc(sizeof(double) * (size_t)(n_seg > 0 ? n_seg : 1) * (size_t)C);
+    skipffn_oracle_summary_forward(X, off, n_seg, C, w, xs, probs);
+    for (int64_t c = 0; c < C; ++c)
+        dw[c] = 0.0;
+    for (int64_t s = 0; s < n_seg; ++s) {
+        const double *g = dxs + s * C;
+        double t = 0.0;
+        for (int64_t i = off[s]; i < off[s + 1]; ++i) {
+            double a = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                a += g[c] * X[i * C + c];
+            t += probs[i] * a;
+        }
+        for (int64_t i = off[s]; i < off[s + 1]; ++i) {
+            double a = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                a += g[c] * X[i * C + c];
+            double ds = probs[i] * (a - t);
+            for (int64_t c = 0; c < C; ++c) {
+                dX[i * C + c] = probs[i] * g[c] + ds * w[c];
+                dw[c] += ds * X[i * C + c];
+            }
+        }
+    }
+    free(probs);
+    free(xs);
+}

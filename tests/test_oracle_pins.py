@@ -387,3 +387,57 @@ def test_prenorm_backward_matches_fp64_autograd_and_finite_differences():
         xp, xm = x.copy(), x.copy()
         xp[t, c] += h; xm[t, c] -= h
         assert abs((loss(xp, gamma) - loss(xm, gamma)) / (2 * h) - got[0][t, c]) < 1e-6
+
+
+# ------------------------------------------------------------------ adaptive summary token (Eq. 6)
+def test_summary_token_special_cases():
+    r = np.random.default_rng(5)
+    X = r.normal(size=(9, 6))
+    off = [0, 4, 4, 5, 9]                     # sizes 4, 0, 1, 4
+    # w = 0: uniform weights, the summary token is the mean of the rows
+    xs, p = oracle.summary_forward(X, off, np.zeros(6))
+    np.testing.assert_allclose(xs[0], X[0:4].mean(0), rtol=1e-14)
+    assert not xs[1].any()                    # empty segment
+    assert xs[2].tolist() == X[4].tolist()    # one row: itself
+    np.testing.assert_allclose(p, [0.25] * 4 + [1.0] + [0.25] * 4)
+    # library softmax
+    from scipy.special import softmax
+    w = r.normal(size=6)
+    xs, p = oracle.summary_forward(X, off, w)
+    for lo, hi, s in [(0, 4, 0), (5, 9, 3)]:
+        q = softmax(X[lo:hi] @ w)
+        np.testing.assert_allclose(p[lo:hi], q, rtol=1e-13)
+        np.testing.assert_allclose(xs[s], q @ X[lo:hi], rtol=1e-13)
+    # a huge score gap selects one row (and the shifted exponent does not overflow)
+    X2 = np.eye(4, 6)
+    xs, p = oracle.summary_forward(X2, [0, 4], np.array([0.0, 0.0, 2000.0, 0.0, 0.0, 0.0]))
+    assert p.tolist() == [0.0, 0.0, 1.0, 0.0] and xs[0].tolist() == X2[2].tolist()
+    # two-row closed form: weights sigmoid(+-d) with d the score difference
+    X3 = np.array([[1.0, 0.0], [0.0, 1.0]])
+    xs, p = oracle.summary_forward(X3, [0, 2], np.array([math.log(3.0), 0.0]))
+    np.testing.assert_allclose(p, [0.75, 0.25], rtol=1e-15)
+    np.testing.assert_allclose(xs[0], [0.75, 0.25], rtol=1e-15)
+
+
+def test_summary_token_backward_autograd_and_finite_differences():
+    import torch
+    r = np.random.default_rng(6)
+    X, w = r.normal(size=(7, 5)), r.normal(size=5)
+    off = [0, 3, 7]
+    dxs = r.normal(size=(2, 5))
+    tX = torch.tensor(X, requires_grad=True)
+    tw = torch.tensor(w, requires_grad=True)
+    ys = [torch.softmax(tX[lo:hi] @ tw, 0) @ tX[lo:hi] for lo, hi in [(0, 3), (3, 7)]]
+    (torch.stack(ys) * torch.tensor(dxs)).sum().backward()
+    dX, dw = oracle.summary_backward(X, off, w, dxs)
+    np.testing.assert_allclose(dX, tX.grad.numpy(), rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(dw, tw.grad.numpy(), rtol=1e-11, atol=1e-13)
+    loss = lambda XX, ww: float(np.sum(dxs * oracle.summary_forward(XX, off, ww)[0]))
+    h = 1e-6
+    for c in range(5):
+        wp, wm = w.copy(), w.copy()
+        wp[c] += h; wm[c] -= h
+        assert abs((loss(X, wp) - loss(X, wm)) / (2 * h) - dw[c]) < 1e-7
+    Xp, Xm = X.copy(), X.copy()
+    Xp[4, 2] += h; Xm[4, 2] -= h
+    assert abs((loss(Xp, w) - loss(Xm, w)) / (2 * h) - dX[4, 2]) < 1e-7
