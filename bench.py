@@ -517,6 +517,57 @@ def run_kv(args):
                                        "sample": f"2 of {planes} planes, {dt * 1e3:.1f} ms"}}), flush=True)
 
 
+# ------------------------------------------------------------------------------ summary token
+def run_summary(args):
+    """Adaptive summary token (Eq. 6) at the cfg2 layout: 8 samples, each with a segment of 144
+    retained and one of 432 skipped visual tokens, C = 4096, bf16; forward + backward."""
+    import torch
+    import oracle
+    import paper_2503_21817_b200 as sk
+    torch.cuda.set_device(0)
+    pk = peaks()
+    C = wl.SWEEP_SHAPES[args.shape][0]
+    sizes = [144, 432] * 8
+    n = sum(sizes)
+    X = wl.round_to(wl.normal(args.seed, wl.TID_X, n * C), "bf16").reshape(n, C)
+    w = wl.round_to(wl.normal(args.seed, wl.TID_WGATE, C, 0.02), "bf16")
+    dxs = wl.round_to(wl.normal(args.seed, wl.TID_DOUT, len(sizes) * C), "bf16").reshape(len(sizes), C)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    bf = lambda a: torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16).reshape(a.shape)
+    Xd, wd, gd, offd = bf(X), bf(w), bf(dxs), torch.from_numpy(off).cuda()
+
+    def step():
+        xs, probs = sk.summary_forward(Xd, offd, wd)
+        return xs, sk.summary_backward(Xd, offd, wd, probs, gd)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        xs, (dX, dw) = step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    moved = 3.0 * n * C * 2              # X read by forward and by backward, dX written
+    t = time.perf_counter()
+    ref_xs, _ = oracle.summary_forward(X[:off[2]], off[:3], w)
+    ref_dX, _ = oracle.summary_backward(X[:off[2]], off[:3], w, dxs[:2])
+    dt = time.perf_counter() - t
+    err = float(np.linalg.norm(xs[:2].float().cpu().numpy() - ref_xs) / np.linalg.norm(ref_xs))
+    gbs = moved / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "summary_token_fwd_bwd_rows_per_s", "value": n / (ms * 1e-3), "unit": "rows/s", "ms": ms,
+                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 8,
+                      "config": {"workload": f"{len(sizes)} segments (8 samples x [144 retained | 432 skipped]), "
+                                             f"{n} rows, C={C}", "l2_policy": "X (38 MB) fits in L2: second reads hit L2"},
+                      "roofline": {"kernel": "summary forward+backward (8 launches)", "bound": "hbm", "achieved": gbs,
+                                   "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
+                                   "peak_source": pk["source"], "traffic": None},
+                      "xs_rel_error_first_sample": err,
+                      "cpu_baseline": {"value": int(off[2]) / dt, "unit": "rows/s", "cores": 1, "kind": "oracle",
+                                       "sample": f"first sample (2 segments, {int(off[2])} rows), {dt:.2f} s"}}), flush=True)
+
+
 # ------------------------------------------------------------------------------ library yardstick
 def run_yardstick(args):
     """Not part of the metric: times the vendor library's plain GEMMs (torch.matmul) on the five
@@ -573,8 +624,11 @@ def main():
     ap.add_argument("--yardstick", action="store_true",
                     help="time the vendor library's plain GEMMs on the path's shapes (context only)")
     ap.add_argument("--kv", action="store_true", help="skip KV-cache compaction (Eq. 7) at the 8B cache shape")
+    ap.add_argument("--summary", action="store_true", help="adaptive summary token (Eq. 6), forward + backward")
     args = ap.parse_args()
-    if args.kv:
+    if args.summary:
+        run_summary(args)
+    elif args.kv:
         run_kv(args)
     elif args.yardstick:
         run_yardstick(args)

@@ -116,6 +116,27 @@ skipffn_status skipffn_forward_prenorm(skipffn_saved *saved, const void *x, cons
 skipffn_status skipffn_backward_prenorm(const void *dout, skipffn_saved *saved, void *dx, void *dgamma,
                                         void *dW_gate, void *dW_up, void *dW_down, void *stream);
 
+/* Adaptive summary token (paper section 4.2, Eq. 6):  x_s = softmax(X w^T)^T X, where X holds the
+ * retained or the skipped visual tokens of one sample and w [C] is the layer's weight.  Needs no
+ * handle.  Several samples are processed at once as segments of a packed X:
+ *   X           : [n_rows, C] device, dtype = skipffn_dtype, C a multiple of 8
+ *   seg_offsets : DEVICE int32 [n_seg + 1], ascending, first 0, last n_rows
+ *   xs          : [n_seg, C] out (an empty segment gives zeros);  probs : [n_rows] fp32 out, the
+ *                 softmax weights, which the backward needs.
+ * Backward for upstream gradient dxs [n_seg, C]: dX [n_rows, C] (may be NULL), dw [C] (may be NULL;
+ * fp32 if dw_fp32 or dtype is fp32), both overwritten.  scratch: device memory of
+ * skipffn_summary_scratch_bytes(n_rows, C) bytes, 16-byte aligned (EWORKSPACE if smaller).
+ * Scores, weights and all sums are fp32 in a fixed order; outputs are rounded once. */
+size_t skipffn_summary_scratch_bytes(int64_t n_rows, int32_t C);
+skipffn_status skipffn_summary_forward(const void *X, const int32_t *seg_offsets, int32_t n_seg,
+                                       int64_t n_rows, int32_t C, int32_t dtype, const void *w,
+                                       void *xs, float *probs, void *stream);
+skipffn_status skipffn_summary_backward(const void *X, const int32_t *seg_offsets, int32_t n_seg,
+                                        int64_t n_rows, int32_t C, int32_t dtype, const void *w,
+                                        const float *probs, const void *dxs, void *dX, void *dw,
+                                        int32_t dw_fp32, void *scratch, size_t scratch_bytes,
+                                        void *stream);
+
 /* Device addresses of the kept-row index list (int32, ascending) and of its length. */
 skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
                                 const int32_t **nk_dev);

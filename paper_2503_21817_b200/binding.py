@@ -18,7 +18,8 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_get_intermediate", "skipffn_poll", "skipffn_last_launches", "skipffn_flops",
            "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
            "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact",
-           "skipffn_forward_prenorm", "skipffn_backward_prenorm"]
+           "skipffn_forward_prenorm", "skipffn_backward_prenorm", "skipffn_summary_scratch_bytes",
+           "skipffn_summary_forward", "skipffn_summary_backward"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
@@ -85,6 +86,13 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_schedule_segment.argtypes = [i32, i32, i32, i32, i32, i32, ctypes.POINTER(i32)]
     lib.skipffn_kv_compact.restype = i32
     lib.skipffn_kv_compact.argtypes = [vp, vp, vp, i64, i64, i64, vp, i32, vp, vp]
+    lib.skipffn_summary_scratch_bytes.restype = ctypes.c_size_t
+    lib.skipffn_summary_scratch_bytes.argtypes = [i64, i32]
+    lib.skipffn_summary_forward.restype = i32
+    lib.skipffn_summary_forward.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp]
+    lib.skipffn_summary_backward.restype = i32
+    lib.skipffn_summary_backward.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, vp, i32, vp,
+                                             ctypes.c_size_t, vp]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -128,6 +136,47 @@ def skipffn_schedule(workers: int, tiles: int, k_blocks: int, split_k: bool, wor
 
 def _ptr(t):
     return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_of(t):
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def summary_forward(X, seg_offsets, w):
+    """Adaptive summary tokens (``skipffn_summary_forward``, Eq. 6).  ``X`` ``[n, C]`` packed rows,
+    ``seg_offsets`` int32 CUDA tensor ``[n_seg + 1]``, ``w`` ``[C]``.  Returns ``(xs [n_seg, C],
+    probs [n] fp32)``; ``probs`` is what the backward needs."""
+    import torch
+    dtype = BF16 if X.dtype == torch.bfloat16 else FP32
+    n, C = X.shape
+    n_seg = seg_offsets.numel() - 1
+    xs = torch.empty(n_seg, C, dtype=X.dtype, device=X.device)
+    probs = torch.empty(max(n, 1), dtype=torch.float32, device=X.device)
+    st = load_library().skipffn_summary_forward(_ptr(X), _ptr(seg_offsets), n_seg, n, C, dtype, _ptr(w), _ptr(xs),
+                                                _ptr(probs), _stream_of(X))
+    if st != 0:
+        raise SkipFFNError(st, "skipffn_summary_forward")
+    return xs, probs[:n]
+
+
+def summary_backward(X, seg_offsets, w, probs, dxs, dw_fp32=False):
+    """``(dX, dw)`` of the adaptive summary layer (``skipffn_summary_backward``)."""
+    import torch
+    lib = load_library()
+    dtype = BF16 if X.dtype == torch.bfloat16 else FP32
+    n, C = X.shape
+    n_seg = seg_offsets.numel() - 1
+    dX = torch.empty_like(X)
+    dw = torch.empty(C, dtype=torch.float32 if (dw_fp32 or dtype == FP32) else X.dtype, device=X.device)
+    nbytes = int(lib.skipffn_summary_scratch_bytes(n, C))
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=X.device)
+    st = lib.skipffn_summary_backward(_ptr(X), _ptr(seg_offsets), n_seg, n, C, dtype, _ptr(w), _ptr(probs),
+                                      _ptr(dxs), _ptr(dX), _ptr(dw), int(dw_fp32), _ptr(scratch), nbytes,
+                                      _stream_of(X))
+    if st != 0:
+        raise SkipFFNError(st, "skipffn_summary_backward")
+    return dX, dw
 
 
 def skipffn_compact_static(skip_mask, idx, nk) -> None:

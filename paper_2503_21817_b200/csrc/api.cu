@@ -440,6 +440,42 @@ skipffn_status skipffn_kv_compact(const skipffn_saved *s, const void *src, void 
     return SKIPFFN_OK;
 }
 
+size_t skipffn_summary_scratch_bytes(int64_t n_rows, int32_t C)
+{
+    if (n_rows < 0 || C <= 0) return 0;
+    return (size_t)(((n_rows + 63) / 64) * 64 + (int64_t)DG_CHUNKS * C) * sizeof(float);
+}
+
+static bool summary_args_ok(const void *X, const int32_t *off, int32_t n_seg, int64_t n_rows, int32_t C,
+                            int32_t dtype, const void *w)
+{
+    return n_seg >= 0 && n_rows >= 0 && n_rows < ((int64_t)1 << 31) && C > 0 && C % 8 == 0 &&
+           (dtype == SKIPFFN_BF16 || dtype == SKIPFFN_FP32) && w && (n_seg == 0 || off) && (n_rows == 0 || X);
+}
+
+skipffn_status skipffn_summary_forward(const void *X, const int32_t *seg_offsets, int32_t n_seg, int64_t n_rows,
+                                       int32_t C, int32_t dtype, const void *w, void *xs, float *probs,
+                                       void *stream)
+{
+    if (!summary_args_ok(X, seg_offsets, n_seg, n_rows, C, dtype, w)) return SKIPFFN_EINVAL;
+    if (n_seg > 0 && (!xs || (n_rows > 0 && !probs))) return SKIPFFN_EINVAL;
+    return launch_summary_forward(X, seg_offsets, n_seg, n_rows, C, dtype, w, xs, probs, (cudaStream_t)stream) ==
+                   cudaSuccess ? SKIPFFN_OK : SKIPFFN_ECUDA;
+}
+
+skipffn_status skipffn_summary_backward(const void *X, const int32_t *seg_offsets, int32_t n_seg, int64_t n_rows,
+                                        int32_t C, int32_t dtype, const void *w, const float *probs,
+                                        const void *dxs, void *dX, void *dw, int32_t dw_fp32, void *scratch,
+                                        size_t scratch_bytes, void *stream)
+{
+    if (!summary_args_ok(X, seg_offsets, n_seg, n_rows, C, dtype, w)) return SKIPFFN_EINVAL;
+    if (n_seg > 0 && (!dxs || !scratch || (n_rows > 0 && !probs))) return SKIPFFN_EINVAL;
+    if (scratch_bytes < skipffn_summary_scratch_bytes(n_rows, C)) return SKIPFFN_EWORKSPACE;
+    if (((uintptr_t)scratch & 15u) != 0) return SKIPFFN_EINVAL;
+    return launch_summary_backward(X, seg_offsets, n_seg, n_rows, C, dtype, w, probs, dxs, dX, dw, dw_fp32,
+                                   (float *)scratch, (cudaStream_t)stream) == cudaSuccess ? SKIPFFN_OK : SKIPFFN_ECUDA;
+}
+
 skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev, const int32_t **nk_dev)
 {
     if (!s || s->planned_N < 0) return SKIPFFN_EINVAL;

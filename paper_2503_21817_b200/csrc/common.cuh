@@ -35,6 +35,32 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// four consecutive elements (C is a multiple of 8, rows are 16-byte aligned)
+__device__ __forceinline__ void load4(const float *p, float (&v)[4])
+{
+    const float4 t = *reinterpret_cast<const float4 *>(p);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void load4(const bf16 *p, float (&v)[4])
+{
+    const uint2 t = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&t.x);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&t.y);
+    v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
+}
+__device__ __forceinline__ void store4(float *p, const float (&v)[4])
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void store4(bf16 *p, const float (&v)[4])
+{
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    uint2 t;
+    t.x = *reinterpret_cast<const uint32_t *>(&a);
+    t.y = *reinterpret_cast<const uint32_t *>(&b);
+    *reinterpret_cast<uint2 *>(p) = t;
+}
+
 __device__ __forceinline__ float sigmoidf_(float z) { return 1.0f / (1.0f + expf(-z)); }
 
 // h = silu(g) * u  (Eq. 4's FFN body, SwiGLU)
@@ -102,6 +128,12 @@ cudaError_t launch_norm_bwd(const float *dY, const void *Xk, const void *dOk, co
                             const int32_t *status, int64_t max_rows, int C, int elem_bytes,
                             int dgamma_fp32, int accumulate, cudaStream_t s);
 constexpr int DG_CHUNKS = 32;   // row chunks of the two-stage dgamma reduction ([DG_CHUNKS, C] fp32 partials)
+// summary.cu
+cudaError_t launch_summary_forward(const void *X, const int32_t *off, int n_seg, int64_t n, int C, int dtype,
+                                   const void *w, void *xs, float *probs, cudaStream_t s);
+cudaError_t launch_summary_backward(const void *X, const int32_t *off, int n_seg, int64_t n, int C, int dtype,
+                                    const void *w, const float *probs, const void *dxs, void *dX, void *dw,
+                                    int dw_fp32, float *scratch, cudaStream_t s);
 // simt.cu
 cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
 // umma.cu (bf16 only)

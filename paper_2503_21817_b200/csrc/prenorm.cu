@@ -11,32 +11,6 @@ namespace skipffn {
 
 constexpr int PN_THREADS = 128;
 
-// four consecutive elements (C is a multiple of 8, rows are 16-byte aligned)
-__device__ __forceinline__ void load4(const float *p, float (&v)[4])
-{
-    const float4 t = *reinterpret_cast<const float4 *>(p);
-    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
-}
-__device__ __forceinline__ void load4(const bf16 *p, float (&v)[4])
-{
-    const uint2 t = *reinterpret_cast<const uint2 *>(p);
-    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&t.x);
-    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&t.y);
-    v[0] = __low2float(a); v[1] = __high2float(a); v[2] = __low2float(b); v[3] = __high2float(b);
-}
-__device__ __forceinline__ void store4(float *p, const float (&v)[4])
-{
-    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
-}
-__device__ __forceinline__ void store4(bf16 *p, const float (&v)[4])
-{
-    const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
-    uint2 t;
-    t.x = *reinterpret_cast<const uint32_t *>(&a);
-    t.y = *reinterpret_cast<const uint32_t *>(&b);
-    *reinterpret_cast<uint2 *>(p) = t;
-}
-
 __device__ __forceinline__ float block_sum(float v, float *red)
 {
 #pragma unroll

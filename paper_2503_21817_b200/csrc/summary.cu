@@ -1,0 +1,202 @@
+// Adaptive summary token (paper section 4.2, Eq. 6):  x_s = softmax(X w^T)^T X  per segment of a
+// packed X [n, C] (the retained or the skipped visual tokens of one sample), w [C].  A tiny layer
+// run once per sample before the decoder; HBM / latency bound.  All sums are fp32 in a fixed order.
+//   forward : scores (one warp per row) -> softmax per segment -> weighted row sum per column block
+//   backward: a_i = dxs . X_i (warp per row) -> ds_i = p_i (a_i - sum_j p_j a_j) per segment
+//             -> dX_i = p_i dxs + ds_i w (rows) and dw = sum_i ds_i X_i (two-stage column reduction)
+#include "common.cuh"
+
+namespace skipffn {
+
+constexpr int SM_THREADS = 256;
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
+// out[i] = sum_c X[i, c] * v[seg(i)?, c]: one warp per row.  per_segment = 0: v is one vector (w);
+// 1: v is [n_seg, C] and the row's segment is found by binary search in the offsets.
+template <typename T>
+__global__ void __launch_bounds__(SM_THREADS)
+k_row_dots(const T *__restrict__ X, const T *__restrict__ v, const int32_t *__restrict__ off, int n_seg,
+           int per_segment, float *__restrict__ out, int64_t n, int C)
+{
+    const int64_t i = (int64_t)blockIdx.x * (SM_THREADS / 32) + (threadIdx.x >> 5);
+    if (i >= n) return;
+    const int lane = threadIdx.x & 31;
+    const T *vec = v;
+    if (per_segment) {
+        int lo = 0, hi = n_seg;            // largest s with off[s] <= i
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (off[mid] <= i) lo = mid; else hi = mid; }
+        vec = v + (int64_t)lo * C;
+    }
+    const T *x = X + i * C;
+    float acc = 0.0f;
+    for (int c = 4 * lane; c < C; c += 128) {    // C is a multiple of 8
+        float a[4], b[4];
+        load4(x + c, a);
+        load4(vec + c, b);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc = fmaf(a[q], b[q], acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) out[i] = acc;
+}
+
+__device__ __forceinline__ float block_reduce(float v, float *red, bool is_max)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        const float o = __shfl_xor_sync(0xffffffffu, v, d);
+        v = is_max ? fmaxf(v, o) : v + o;
+    }
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int w = 1; w < SM_THREADS / 32; ++w) r = is_max ? fmaxf(r, red[w]) : r + red[w];
+    return r;
+}
+
+// probs[i] <- softmax of the scores in probs, per segment (one CTA per segment, in place)
+__global__ void __launch_bounds__(SM_THREADS)
+k_segment_softmax(float *__restrict__ probs, const int32_t *__restrict__ off)
+{
+    __shared__ float red[SM_THREADS / 32];
+    const int lo = off[blockIdx.x], hi = off[blockIdx.x + 1];
+    float mx = -INFINITY;
+    for (int i = lo + threadIdx.x; i < hi; i += SM_THREADS) mx = fmaxf(mx, probs[i]);
+    mx = block_reduce(mx, red, true);
+    float den = 0.0f;
+    for (int i = lo + threadIdx.x; i < hi; i += SM_THREADS) den += expf(probs[i] - mx);
+    den = block_reduce(den, red, false);
+    for (int i = lo + threadIdx.x; i < hi; i += SM_THREADS) probs[i] = expf(probs[i] - mx) / den;
+}
+
+// a[i] <- ds_i = p_i (a_i - sum_j p_j a_j), per segment, in place
+__global__ void __launch_bounds__(SM_THREADS)
+k_segment_dscore(float *__restrict__ a, const float *__restrict__ probs, const int32_t *__restrict__ off)
+{
+    __shared__ float red[SM_THREADS / 32];
+    const int lo = off[blockIdx.x], hi = off[blockIdx.x + 1];
+    float t = 0.0f;
+    for (int i = lo + threadIdx.x; i < hi; i += SM_THREADS) t = fmaf(probs[i], a[i], t);
+    t = block_reduce(t, red, false);
+    for (int i = lo + threadIdx.x; i < hi; i += SM_THREADS) a[i] = probs[i] * (a[i] - t);
+}
+
+// y[c] = sum over rows lo..hi-1 of coef[i] * X[i, c]; grid (column blocks of 64, parts); 4 row lanes
+// per column, combined in lane order.  parts == n_seg with seg_mode (rows of segment blockIdx.y,
+// output xs[seg]), else DG_CHUNKS equal chunks of all rows (output part[chunk]).
+constexpr int SP_COLS = 64, SP_LANES = 8;
+
+template <typename T, typename TO>
+__global__ void __launch_bounds__(SP_COLS * SP_LANES)
+k_weighted_rows(const T *__restrict__ X, const float *__restrict__ coef, const int32_t *__restrict__ off,
+                int seg_mode, int64_t n, TO *__restrict__ out, int C)
+{
+    __shared__ float red[SP_LANES][SP_COLS];
+    int64_t lo, hi;
+    if (seg_mode) { lo = off[blockIdx.y]; hi = off[blockIdx.y + 1]; }
+    else { const int64_t per = (n + gridDim.y - 1) / gridDim.y; lo = blockIdx.y * per; hi = lo + per < n ? lo + per : n; }
+    const int cl = threadIdx.x % SP_COLS, lane = threadIdx.x / SP_COLS;
+    const int col = blockIdx.x * SP_COLS + cl;
+    float acc = 0.0f;
+    if (col < C) {
+#pragma unroll 8
+        for (int64_t i = lo + lane; i < hi; i += SP_LANES) acc = fmaf(coef[i], to_f32(X[i * C + col]), acc);
+    }
+    red[lane][cl] = acc;
+    __syncthreads();
+    if (lane == 0 && col < C) {
+        float s = 0.0f;
+#pragma unroll
+        for (int l = 0; l < SP_LANES; ++l) s += red[l][cl];
+        out[(int64_t)blockIdx.y * C + col] = from_f32<TO>(s);
+    }
+}
+
+template <typename TO>
+__global__ void k_sum_parts(const float *__restrict__ part, int parts, TO *__restrict__ out, int C)
+{
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    if (col >= C) return;
+    float s = 0.0f;
+    for (int k = 0; k < parts; ++k) s += part[(int64_t)k * C + col];
+    out[col] = from_f32<TO>(s);
+}
+
+// dX[i, c] = p_i * dxs[seg(i), c] + ds_i * w[c]: one CTA per row
+template <typename T>
+__global__ void __launch_bounds__(SM_THREADS)
+k_summary_dx(const T *__restrict__ dxs, const T *__restrict__ w, const float *__restrict__ probs,
+             const float *__restrict__ ds, const int32_t *__restrict__ off, int n_seg, T *__restrict__ dX, int C)
+{
+    const int64_t i = blockIdx.x;
+    int lo = 0, hi = n_seg;
+    while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (off[mid] <= i) lo = mid; else hi = mid; }
+    const T *g = dxs + (int64_t)lo * C;
+    const float p = probs[i], d = ds[i];
+    for (int c = threadIdx.x; c < C; c += SM_THREADS)
+        dX[i * C + c] = from_f32<T>(fmaf(p, to_f32(g[c]), d * to_f32(w[c])));
+}
+
+template <typename T>
+static cudaError_t fwd_t(const T *X, const int32_t *off, int n_seg, int64_t n, int C, const T *w, T *xs,
+                         float *probs, cudaStream_t s)
+{
+    if (n > 0) {
+        k_row_dots<T><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, w, off, n_seg, 0, probs, n, C);
+        k_segment_softmax<<<n_seg, SM_THREADS, 0, s>>>(probs, off);
+    }
+    dim3 grid((C + SP_COLS - 1) / SP_COLS, n_seg);     // empty segments write zeros
+    k_weighted_rows<T, T><<<grid, SP_COLS * SP_LANES, 0, s>>>(X, probs, off, 1, n, xs, C);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t bwd_t(const T *X, const int32_t *off, int n_seg, int64_t n, int C, const T *w,
+                         const float *probs, const T *dxs, T *dX, void *dw, int dw_fp32, float *scratch,
+                         cudaStream_t s)
+{
+    float *ds = scratch, *part = scratch + ((n + 63) / 64) * 64;
+    if (n > 0) {
+        k_row_dots<T><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, dxs, off, n_seg, 1, ds, n, C);
+        k_segment_dscore<<<n_seg, SM_THREADS, 0, s>>>(ds, probs, off);
+        if (dX) k_summary_dx<T><<<(unsigned)n, SM_THREADS, 0, s>>>(dxs, w, probs, ds, off, n_seg, dX, C);
+    }
+    if (dw) {
+        dim3 grid((C + SP_COLS - 1) / SP_COLS, DG_CHUNKS);
+        k_weighted_rows<T, float><<<grid, SP_COLS * SP_LANES, 0, s>>>(X, ds, off, 0, n, part, C);
+        if (dw_fp32) k_sum_parts<float><<<(C + 255) / 256, 256, 0, s>>>(part, DG_CHUNKS, (float *)dw, C);
+        else k_sum_parts<T><<<(C + 255) / 256, 256, 0, s>>>(part, DG_CHUNKS, (T *)dw, C);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_summary_forward(const void *X, const int32_t *off, int n_seg, int64_t n, int C, int dtype,
+                                   const void *w, void *xs, float *probs, cudaStream_t s)
+{
+    if (n_seg <= 0) return cudaSuccess;
+    return dtype == SKIPFFN_BF16
+               ? fwd_t<bf16>((const bf16 *)X, off, n_seg, n, C, (const bf16 *)w, (bf16 *)xs, probs, s)
+               : fwd_t<float>((const float *)X, off, n_seg, n, C, (const float *)w, (float *)xs, probs, s);
+}
+
+cudaError_t launch_summary_backward(const void *X, const int32_t *off, int n_seg, int64_t n, int C, int dtype,
+                                    const void *w, const float *probs, const void *dxs, void *dX, void *dw,
+                                    int dw_fp32, float *scratch, cudaStream_t s)
+{
+    if (n_seg <= 0) return cudaSuccess;
+    return dtype == SKIPFFN_BF16
+               ? bwd_t<bf16>((const bf16 *)X, off, n_seg, n, C, (const bf16 *)w, probs, (const bf16 *)dxs,
+                             (bf16 *)dX, dw, dw_fp32, scratch, s)
+               : bwd_t<float>((const float *)X, off, n_seg, n, C, (const float *)w, probs, (const float *)dxs,
+                              (float *)dX, dw, 1, scratch, s);
+}
+
+}  // namespace skipffn
