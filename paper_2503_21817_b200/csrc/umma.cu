@@ -328,6 +328,7 @@ struct UmmaParams {
     float4 *sk_slots;                // per-CTA partial-accumulator slots
     int32_t *sk_flags;               // SK_FLAGS_PER_CTA flags per slot
     int32_t sk_epoch;                // flag value of this launch
+    int32_t sk_wait_skew;            // 0; test hook: finishing units wait for a value nobody writes
     // grouped launch (weight gradients): up to three independent problems sharing K; problem g has
     // extents gM[g] x gN[g], operands (tmA, tmB) / (tmA2, tmB2) / (tmA3, tmB2), output gout[g]
     int32_t groups;
@@ -712,8 +713,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 // the rest of this tile's K range sits in the slots of workers src_lo .. worker-1
                 for (int q = sg.src_lo; ok && q < worker; ++q) {
                     if (sched.bound(q + 1) == sched.bound(q)) continue;   // that worker had no run
-                    ok = flag_wait(p.sk_flags + (q * SPLIT + (int)rank) * SK_FLAGS_PER_CTA + ew, p.sk_epoch,
-                                   lane, abort_flag, p.status);
+                    ok = flag_wait(p.sk_flags + (q * SPLIT + (int)rank) * SK_FLAGS_PER_CTA + ew,
+                                   p.sk_epoch + p.sk_wait_skew, lane, abort_flag, p.status);
                 }
                 if (!ok) break;
             }
@@ -1049,6 +1050,11 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_slots = (float4 *)g.sk_slots;
     p.sk_flags = g.sk_flags;
     p.sk_epoch = g.sk_epoch;
+    // Test hook for the failure path: with SKIPFFN_TEST_LOST_HANDOVER set, units that finish a tile
+    // wait for a hand-over flag value that no producer writes, so their bounded wait runs out, the
+    // kernel records SKIPFFN_ETIMEOUT (site SITE_EPI_PARTIAL) and returns normally after about 1 s.
+    p.sk_wait_skew = 0;
+    if (const char *e = getenv("SKIPFFN_TEST_LOST_HANDOVER")) { if (atoi(e) != 0) p.sk_wait_skew = 0x40000000; }
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
     static const int sk_threshold[5] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40};
     p.streamk = (g.sk_slots && g.sk_flags) ? sk_threshold[epi] : 0;

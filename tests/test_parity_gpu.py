@@ -349,3 +349,27 @@ def test_sweep_end_points_vicuna_13b_shape_sampled(ratio):
         check(to_host(r["dW_down"][:, cols].T), c, "bf16", "dW_down cols")
         idx, nk = r["ctx"].kept()
         assert nk == w.N and np.array_equal(idx.cpu().numpy(), np.arange(w.N))
+
+
+def test_lost_hand_over_is_reported_and_the_context_stays_usable(monkeypatch):
+    # Failure path without a fault: with the test hook set, units that finish a K-split tile wait
+    # for a hand-over that never comes.  The wait is bounded (about 1 s): the kernel must return,
+    # skipffn_poll must report SKIPFFN_ETIMEOUT with the hand-over site, and the same handle must
+    # then produce correct results again.
+    import time
+    sk = _sk()
+    w = wl.small_case(25, "bf16", 256, 4096, 2, 16, 200, 0.5)
+    dev = DeviceWorkload(w)
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    monkeypatch.setenv("SKIPFFN_STREAMK", "1")             # cut along K whenever tiles do not fill a wave
+    monkeypatch.setenv("SKIPFFN_TEST_LOST_HANDOVER", "1")
+    t0 = time.time()
+    ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
+    with pytest.raises(sk.SkipFFNError) as e:
+        ctx.poll()
+    assert e.value.status == 5 and "site 6" in str(e.value)
+    assert time.time() - t0 < 30
+    monkeypatch.delenv("SKIPFFN_TEST_LOST_HANDOVER")
+    out = ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
+    ctx.poll()                                              # status word was cleared by the failed poll
+    check(to_host(out), oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down), "bf16", "out after recovery")
