@@ -399,6 +399,31 @@ __device__ __forceinline__ void store_rows_64B(uint32_t sbuf, int lane, const ui
     }
     __syncwarp();
 }
+// The reverse for epilogue inputs.  `v[it]` holds the 16 bytes this lane loaded from row
+// it * 8 + lane / 4, slot lane % 4 (four consecutive lanes cover one row's 64 bytes, so a warp
+// load touches eight full 64-byte segments instead of 32 scattered 16-byte pieces); the same
+// staging buffer turns them into this lane's own row as 16 packed words.
+__device__ __forceinline__ void rows_from_coalesced(uint32_t sbuf, int lane, const uint4 (&v)[4],
+                                                    uint32_t (&w)[16])
+{
+    const int c = lane & 3;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = it * 8 + (lane >> 2);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + row * 64 + ((c ^ ((row >> 1) & 3)) << 4)),
+                     "r"(v[it].x), "r"(v[it].y), "r"(v[it].z), "r"(v[it].w)
+                     : "memory");
+    }
+    __syncwarp();
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(w[4 * q]), "=r"(w[4 * q + 1]), "=r"(w[4 * q + 2]), "=r"(w[4 * q + 3])
+                     : "r"(sbuf + lane * 64 + ((q ^ sw) << 4))
+                     : "memory");
+    __syncwarp();
+}
 // fp32 variant with read-modify-write (dW accumulation): same staging, 16 columns per call
 __device__ __forceinline__ void store_rows_64B_f32(uint32_t sbuf, int lane, const uint32_t (&w)[16],
                                                    char *my_row, int valid_slots, int accumulate)
@@ -688,15 +713,18 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             // prefetch of the per-row epilogue inputs of the first chunk (overlaps the accumulator wait)
             uint4 pa[4], pb[4];
             auto prefetch = [&](int n) {
+                // compact rows m0 + quarter * 32 .. + 31 of in0 / in1, loaded eight rows per instruction
                 if ((EPI == EPI_DH || EPI == EPI_DOWN || EPI == EPI_DX) && p.in0 != nullptr) {
-                    const int64_t o = (int64_t)m * p.ldo + n;
+                    const int c = lane & 3;
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        pa[v] = make_uint4(0, 0, 0, 0);
-                        pb[v] = make_uint4(0, 0, 0, 0);
-                        if (row_valid && n + v * 8 < n_end) {
-                            pa[v] = reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o)[v];
-                            if (EPI == EPI_DH) pb[v] = reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o)[v];
+                    for (int it = 0; it < 4; ++it) {
+                        const int mr = m0 + quarter * 32 + it * 8 + (lane >> 2);
+                        pa[it] = make_uint4(0, 0, 0, 0);
+                        pb[it] = make_uint4(0, 0, 0, 0);
+                        if (mr < pick(g_m, tl.g) && n + c * 8 < n_end) {
+                            const int64_t o = (int64_t)mr * p.ldo + n + c * 8;
+                            pa[it] = __ldcs(reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o));
+                            if (EPI == EPI_DH) pb[it] = __ldcs(reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o));
                         }
                     }
                 }
@@ -797,8 +825,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
                     // residual add in fp32, one rounding, scatter to the token's row
-                    const uint32_t rw[16] = {ca[0].x, ca[0].y, ca[0].z, ca[0].w, ca[1].x, ca[1].y, ca[1].z, ca[1].w,
-                                             ca[2].x, ca[2].y, ca[2].z, ca[2].w, ca[3].x, ca[3].y, ca[3].z, ca[3].w};
+                    uint32_t rw[16];
+                    rows_from_coalesced(sbuf, lane, ca, rw);
 #pragma unroll
                     for (int q = 0; q < 16; ++q) {
                         float a0, a1;
@@ -808,10 +836,9 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     char *row = row_valid ? (char *)((bf16 *)p.out0 + tok * p.ldo + n) : nullptr;
                     store_rows_64B(sbuf, lane, w, row, valid_slots);
                 } else if (EPI == EPI_DH) {
-                    const uint32_t gw[16] = {ca[0].x, ca[0].y, ca[0].z, ca[0].w, ca[1].x, ca[1].y, ca[1].z, ca[1].w,
-                                             ca[2].x, ca[2].y, ca[2].z, ca[2].w, ca[3].x, ca[3].y, ca[3].z, ca[3].w};
-                    const uint32_t uw[16] = {cb[0].x, cb[0].y, cb[0].z, cb[0].w, cb[1].x, cb[1].y, cb[1].z, cb[1].w,
-                                             cb[2].x, cb[2].y, cb[2].z, cb[2].w, cb[3].x, cb[3].y, cb[3].z, cb[3].w};
+                    uint32_t gw[16], uw[16];
+                    rows_from_coalesced(sbuf, lane, ca, gw);
+                    rows_from_coalesced(sbuf, lane, cb, uw);
                     uint32_t w2[16];
 #pragma unroll
                     for (int q = 0; q < 16; ++q) {
