@@ -379,7 +379,7 @@ def run_ours(args):
         roofline["all_gemm_kernels"]["frac"] = roofline["all_gemm_kernels"]["tflops"] / pk["bf16_tflops"]
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:    # the oracle is timed at N = 1 only
         rate, kept, dt, cores = oracle_sample_rate(w, args.cpu_sample_tokens)
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"first {args.cpu_sample_tokens} tokens of sequence 0 ({kept} kept), full fp64 "

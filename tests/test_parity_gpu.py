@@ -373,3 +373,35 @@ def test_lost_hand_over_is_reported_and_the_context_stays_usable(monkeypatch):
     out = ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
     ctx.poll()                                              # status word was cleared by the failed poll
     check(to_host(out), oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down), "bf16", "out after recovery")
+
+
+def test_single_cta_launch_shape_in_a_fresh_process():
+    # The one-CTA-per-tile shape (used when SM pairs cannot be co-scheduled) is chosen once per
+    # process, so it is exercised in a child process: the tiny, ragged, K-split and grouped cases.
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, SKIPFFN_SINGLE_CTA="1")
+    here = os.path.abspath(__file__)
+    p = subprocess.run([sys.executable, "-m", "pytest", here, "-m", "gpu", "-x", "-q", "-k",
+                        "config1_tiny or multi_tile_ragged or k_split_schedule or kept_count_edges or fp32_gradients"],
+                       env=env, capture_output=True, text=True, timeout=900)
+    assert p.returncode == 0, p.stdout[-3000:] + p.stderr[-2000:]
+    assert " passed" in p.stdout
+
+
+def test_bf16_gradient_accumulation():
+    # dW += ... with bf16 gradients: the fp32 tile is added to the stored value and rounded once
+    import torch
+    w = wl.small_case(41, "bf16", 256, 512, 2, 16, 120, 0.7)
+    ref = _oracle_all(w)
+    init = [torch.full((w.I, w.C), 0.5, device="cuda", dtype=torch.bfloat16),
+            torch.full((w.I, w.C), -0.25, device="cuda", dtype=torch.bfloat16),
+            torch.full((w.C, w.I), 1.0, device="cuda", dtype=torch.bfloat16)]
+    r = run(w, accumulate_dw=True, dw_init=[t.clone() for t in init])
+    for k, t in zip(("dW_gate", "dW_up", "dW_down"), init):
+        want = ref[k] + float(t[0, 0])
+        got = to_host(r[k])
+        # one bf16 rounding of a value near |init|: absolute error below half an ulp of the sum
+        assert np.max(np.abs(got - want)) <= 2.0 ** -8 * np.max(np.abs(want)) + 3e-2 * np.sqrt(np.mean(ref[k] ** 2))
+        assert abs(np.mean(got - want)) < 1e-3
