@@ -57,6 +57,10 @@ def _load() -> ctypes.CDLL:
         lib.skipffn_oracle_summary_forward.argtypes = [dp, ctypes.c_void_p, i64, i64, dp, dp, dp]
         lib.skipffn_oracle_summary_backward.restype = None
         lib.skipffn_oracle_summary_backward.argtypes = [dp, ctypes.c_void_p, i64, i64, dp, dp, dp, dp]
+        lib.skipffn_oracle_token_merge.restype = None
+        lib.skipffn_oracle_token_merge.argtypes = [dp, i64, i64, i64, dp, ctypes.c_void_p, ctypes.c_void_p, dp]
+        lib.skipffn_oracle_merge_given.restype = None
+        lib.skipffn_oracle_merge_given.argtypes = [dp, i64, i64, i64, ctypes.c_void_p, dp]
         lib.skipffn_oracle_kv_compact.restype = i64
         lib.skipffn_oracle_kv_compact.argtypes = [bp, bp, i64, i64, i64, bp]
         lib.skipffn_oracle_kept_cu_seqlens.restype = None
@@ -225,3 +229,26 @@ def summary_backward(X, offsets, w, dxs):
     dw = np.empty(C, dtype=np.float64)
     _load().skipffn_oracle_summary_backward(_p(X), _p(off), off.size - 1, C, _p(w), _p(dxs), _p(dX), _p(dw))
     return dX, dw
+
+
+def token_merge(X, k):
+    """Token merge of section 4.1: ``(avg [n], kept [k], assign [n], merged [k, C])``."""
+    X = _f64(X)
+    n, C = X.shape
+    assert 0 < k <= n
+    avg = np.empty(n, dtype=np.float64)
+    kept = np.empty(k, dtype=np.int32)
+    assign = np.empty(n, dtype=np.int32)
+    merged = np.empty((k, C), dtype=np.float64)
+    _load().skipffn_oracle_token_merge(_p(X), n, C, k, _p(avg), _p(kept), _p(assign), _p(merged))
+    return avg, kept, assign, merged
+
+
+def merge_given(X, k, assign):
+    """Mean of the rows assigned to each of the k groups."""
+    X = _f64(X)
+    a = np.ascontiguousarray(assign, dtype=np.int32)
+    n, C = X.shape
+    merged = np.empty((k, C), dtype=np.float64)
+    _load().skipffn_oracle_merge_given(_p(X), n, C, k, _p(a), _p(merged))
+    return merged

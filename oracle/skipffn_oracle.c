@@ -403,3 +403,96 @@ void skipffn_oracle_summary_backward(const double *X, const int32_t *off, int64_
     free(probs);
     free(xs);
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Token merge of the skipped tokens (section 4.1, three steps):
+ *   1. cosine similarity between every pair of tokens; an average similarity per token;
+ *   2. keep the k tokens with the LOWEST average similarity (the most distinctive ones);
+ *   3. merge each of the other n-k tokens into the most similar kept token.
+ * Readings where the paper is silent: the average runs over all n tokens including the token
+ * itself (leaving it out is a monotone change, so the order is the same); ties in step 2 go to
+ * the lower token index; the kept tokens are listed in ascending token order; ties in step 3 go
+ * to the first kept token in that list; the merge operator is NOT stated in the paper -- this
+ * oracle takes the mean of the kept token and everything merged into it ("parity unpinned" for
+ * that operator; steps 1-3 are pinned by brute force and closed forms).
+ * Outputs: avg[n]; kept[k] ascending token indices; assign[n] = position in `kept` of the token's
+ * target (a kept token maps to itself); merged[k, C].  A zero row has similarity 0 with everything.
+ */
+void skipffn_oracle_token_merge(const double *X, int64_t n, int64_t C, int64_t k, double *avg,
+                                int32_t *kept, int32_t *assign, double *merged)
+{
+    double *rn = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    for (int64_t i = 0; i < n; ++i) {
+        double ss = 0.0;
+        for (int64_t c = 0; c < C; ++c)
+            ss += X[i * C + c] * X[i * C + c];
+        rn[i] = ss > 0.0 ? 1.0 / sqrt(ss) : 0.0;
+    }
+    for (int64_t i = 0; i < n; ++i) {
+        double s = 0.0;
+        for (int64_t j = 0; j < n; ++j) {
+            double d = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                d += X[i * C + c] * X[j * C + c];
+            s += d * rn[i] * rn[j];
+        }
+        avg[i] = s / (double)n;
+    }
+    /* rank by (avg, index); keep ranks 0..k-1, listed by ascending index */
+    int64_t nk = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t rank = 0;
+        for (int64_t j = 0; j < n; ++j)
+            if (avg[j] < avg[i] || (avg[j] == avg[i] && j < i))
+                ++rank;
+        if (rank < k)
+            kept[nk++] = (int32_t)i;
+    }
+    double *cnt = (double *)malloc(sizeof(double) * (size_t)(k > 0 ? k : 1));
+    for (int64_t j = 0; j < k; ++j) {
+        cnt[j] = 1.0;
+        assign[kept[j]] = (int32_t)j;
+        for (int64_t c = 0; c < C; ++c)
+            merged[j * C + c] = X[(int64_t)kept[j] * C + c];
+    }
+    for (int64_t i = 0, q = 0; i < n; ++i) {
+        if (q < k && kept[q] == i) { ++q; continue; } /* a kept token */
+        int64_t best = 0;
+        double best_s = -INFINITY;
+        for (int64_t j = 0; j < k; ++j) {
+            double d = 0.0;
+            for (int64_t c = 0; c < C; ++c)
+                d += X[i * C + c] * X[(int64_t)kept[j] * C + c];
+            d *= rn[i] * rn[kept[j]];
+            if (d > best_s) { best_s = d; best = j; }
+        }
+        assign[i] = (int32_t)best;
+        cnt[best] += 1.0;
+        for (int64_t c = 0; c < C; ++c)
+            merged[best * C + c] += X[i * C + c];
+    }
+    for (int64_t j = 0; j < k; ++j)
+        for (int64_t c = 0; c < C; ++c)
+            merged[j * C + c] /= cnt[j];
+    free(rn);
+    free(cnt);
+}
+
+/* The merge operator alone, for a given assignment (used to compare merged rows when the
+ * assignment itself was decided elsewhere): mean over {t : assign[t] == j}. */
+void skipffn_oracle_merge_given(const double *X, int64_t n, int64_t C, int64_t k, const int32_t *assign,
+                                double *merged)
+{
+    double *cnt = (double *)calloc((size_t)(k > 0 ? k : 1), sizeof(double));
+    for (int64_t j = 0; j < k * C; ++j)
+        merged[j] = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        cnt[assign[i]] += 1.0;
+        for (int64_t c = 0; c < C; ++c)
+            merged[(int64_t)assign[i] * C + c] += X[i * C + c];
+    }
+    for (int64_t j = 0; j < k; ++j)
+        for (int64_t c = 0; c < C; ++c)
+            merged[j * C + c] /= (cnt[j] > 0.0 ? cnt[j] : 1.0);
+    free(cnt);
+}

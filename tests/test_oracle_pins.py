@@ -441,3 +441,40 @@ def test_summary_token_backward_autograd_and_finite_differences():
     Xp, Xm = X.copy(), X.copy()
     Xp[4, 2] += h; Xm[4, 2] -= h
     assert abs((loss(Xp, w) - loss(Xm, w)) / (2 * h) - dX[4, 2]) < 1e-7
+
+
+# ------------------------------------------------------------------ token merge (section 4.1)
+def test_token_merge_bruteforce_and_hand_case():
+    r = np.random.default_rng(8)
+    X = r.normal(size=(13, 6))
+    k = 4
+    avg, kept, assign, merged = oracle.token_merge(X, k)
+    Xh = X / np.linalg.norm(X, axis=1, keepdims=True)
+    S = Xh @ Xh.T                                            # library routine
+    np.testing.assert_allclose(avg, S.mean(1), rtol=1e-12)
+    want_kept = sorted(np.argsort(S.mean(1), kind="stable")[:k].tolist())
+    assert kept.tolist() == want_kept
+    for i in range(13):
+        if i in want_kept:
+            assert kept[assign[i]] == i
+        else:
+            assert assign[i] == int(np.argmax(S[i, want_kept]))
+    for j in range(k):
+        members = [i for i in range(13) if assign[i] == j]
+        np.testing.assert_allclose(merged[j], X[members].mean(0), rtol=1e-12)
+    np.testing.assert_allclose(oracle.merge_given(X, k, assign), merged, rtol=1e-13)
+    # hand case in the plane: e1, e1 (duplicate), e2, -e1.  S rows sum to (1, 1, 1, -1): the
+    # most distinctive token is -e1 (average -1/4); next, by index, token 0.
+    X = np.array([[1.0, 0.0], [2.0, 0.0], [0.0, 3.0], [-1.0, 0.0]])
+    avg, kept, assign, merged = oracle.token_merge(X, 2)
+    assert avg.tolist() == [0.25, 0.25, 0.25, -0.25]
+    assert kept.tolist() == [0, 3]
+    assert assign.tolist() == [0, 0, 0, 1]                   # e2 is orthogonal to both: tie -> first
+    assert merged.tolist() == [[1.0, 1.0], [-1.0, 0.0]]
+    # k = n keeps everything unchanged
+    avg, kept, assign, merged = oracle.token_merge(X, 4)
+    assert kept.tolist() == [0, 1, 2, 3] and assign.tolist() == [0, 1, 2, 3] and np.array_equal(merged, X)
+    # average similarity without the full matrix: dot with the mean unit vector (used as a closed form)
+    Y = r.normal(size=(40, 9))
+    Yh = Y / np.linalg.norm(Y, axis=1, keepdims=True)
+    np.testing.assert_allclose(oracle.token_merge(Y, 5)[0], Yh @ Yh.mean(0), rtol=1e-12)
