@@ -568,6 +568,48 @@ def run_summary(args):
                                        "sample": f"first sample (2 segments, {int(off[2])} rows), {dt:.2f} s"}}), flush=True)
 
 
+# ------------------------------------------------------------------------------ token merge
+def run_merge(args):
+    """Token merge (section 4.1) of one high-resolution sample: 2304 skipped tokens merged into 288."""
+    import torch
+    import oracle
+    import paper_2503_21817_b200 as sk
+    torch.cuda.set_device(0)
+    pk = peaks()
+    C = wl.SWEEP_SHAPES[args.shape][0]
+    n, k, clusters = 2304, 288, 64
+    centers = wl.normal(args.seed, wl.TID_WGATE, clusters * C).reshape(clusters, C)
+    which = (wl.raw_u64(args.seed, wl.TID_LAYOUT, 0, n) % np.uint64(clusters)).astype(np.int64)
+    X = wl.round_to(centers[which] + 0.35 * wl.normal(args.seed, wl.TID_X, n * C).reshape(n, C), "bf16")
+    Xd = torch.from_numpy(wl.to_bf16_bits(X).view(np.int16)).cuda().view(torch.bfloat16).reshape(n, C)
+    for _ in range(max(args.warmup, 3)):
+        sk.token_merge(Xd, k)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        kept, assign, merged = sk.token_merge(Xd, k)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    ns = 256                                           # oracle on a bounded sample: the first 256 tokens, 32 kept
+    t = time.perf_counter()
+    oracle.token_merge(X[:ns].astype(np.float64), 32)
+    dt = time.perf_counter() - t
+    flops = 2.0 * (n - k) * k * C + 4.0 * n * C
+    moved = (4.0 * n + k) * C * 2                      # X read by norms, mean, averages, gather and merge
+    print(json.dumps({"metric": "token_merge_rows_per_s", "value": n / (ms * 1e-3), "unit": "rows/s", "ms": ms,
+                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 13,
+                      "config": {"workload": f"{n} tokens of {clusters} noisy clusters, C={C}, keep {k}",
+                                 "l2_policy": "X (19 MB) stays in L2 after the first pass"},
+                      "roofline": {"kernel": "token merge (13 launches)", "bound": "hbm",
+                                   "achieved": moved / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                                   "frac": moved / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "peak_source": pk["source"],
+                                   "traffic": None, "gemm_tflops": flops / (ms * 1e-3) / 1e12},
+                      "cpu_baseline": {"value": ns / dt, "unit": "rows/s", "cores": 1, "kind": "oracle",
+                                       "sample": f"first {ns} tokens, keep 32, {dt:.2f} s"}}), flush=True)
+
+
 # ------------------------------------------------------------------------------ library yardstick
 def run_yardstick(args):
     """Not part of the metric: times the vendor library's plain GEMMs (torch.matmul) on the five
@@ -625,8 +667,11 @@ def main():
                     help="time the vendor library's plain GEMMs on the path's shapes (context only)")
     ap.add_argument("--kv", action="store_true", help="skip KV-cache compaction (Eq. 7) at the 8B cache shape")
     ap.add_argument("--summary", action="store_true", help="adaptive summary token (Eq. 6), forward + backward")
+    ap.add_argument("--merge", action="store_true", help="token merge of section 4.1 on one high-resolution sample")
     args = ap.parse_args()
-    if args.summary:
+    if args.merge:
+        run_merge(args)
+    elif args.summary:
         run_summary(args)
     elif args.kv:
         run_kv(args)

@@ -137,6 +137,29 @@ skipffn_status skipffn_summary_backward(const void *X, const int32_t *seg_offset
                                         int32_t dw_fp32, void *scratch, size_t scratch_bytes,
                                         void *stream);
 
+/* Token merge of the skipped visual tokens (paper section 4.1): (1) cosine similarity between every
+ * pair of the n tokens and an average similarity per token, (2) the k tokens with the LOWEST average
+ * are kept, (3) each other token is merged into its most similar kept token.
+ *   X      : [n, C] device, dtype = skipffn_dtype; C a multiple of 8, at most 16384; n <= 65536
+ *   k      : tokens to keep, a multiple of 4, 1 <= k <= n
+ *   kept   : [k] int32 out, the kept tokens' indices in ascending order
+ *   assign : [n] int32 out, for every token the position in `kept` of the token it goes to (a kept
+ *            token goes to itself)
+ *   merged : [k, C] out, dtype as X
+ *   scratch: device memory of skipffn_token_merge_scratch_bytes(...) bytes, 256-byte aligned.
+ * Where the paper is silent: the average includes the token itself (leaving it out would not change
+ * the order); equal averages go to the lower index; equal similarities in (3) go to the first kept
+ * token; a zero row has similarity 0 with everything; the MERGE OPERATOR IS NOT STATED in the paper
+ * and is taken as the mean of a kept token and the tokens merged into it, summed in token order.
+ * The average is computed as the dot product with the mean unit vector (no n x n matrix); the
+ * (n-k) x k similarity matrix of step (3) runs on the tensor cores for bf16, on unit rows rounded
+ * to bf16.  Statistics are fp32; decisions between nearly equal values may differ from an
+ * exact-arithmetic evaluation. */
+size_t skipffn_token_merge_scratch_bytes(int64_t n, int32_t C, int32_t k, int32_t dtype);
+skipffn_status skipffn_token_merge(const void *X, int64_t n, int32_t C, int32_t k, int32_t dtype,
+                                   int32_t *kept, int32_t *assign, void *merged, void *scratch,
+                                   size_t scratch_bytes, void *stream);
+
 /* Device addresses of the kept-row index list (int32, ascending) and of its length. */
 skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
                                 const int32_t **nk_dev);

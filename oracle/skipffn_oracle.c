@@ -1,5 +1,7 @@
 /*
  * Skip-FFN reference oracle -- TEST INFRASTRUCTURE, not part of the product.
+ * (Parity unpinned: the merge OPERATOR of skipffn_oracle_token_merge / skipffn_oracle_merge_given,
+ * which the paper does not define; everything else below is pinned.)
  *
  * A plain, slow, obviously-correct CPU statement of what the Skip-FFN decoder
  * sublayer computes, forward and backward, in double precision.  It shares no

@@ -19,7 +19,8 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_strerror", "skipffn_profile_enable", "skipffn_profile_read",
            "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact",
            "skipffn_forward_prenorm", "skipffn_backward_prenorm", "skipffn_summary_scratch_bytes",
-           "skipffn_summary_forward", "skipffn_summary_backward"]
+           "skipffn_summary_forward", "skipffn_summary_backward", "skipffn_token_merge_scratch_bytes",
+           "skipffn_token_merge"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
@@ -93,6 +94,10 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_summary_backward.restype = i32
     lib.skipffn_summary_backward.argtypes = [vp, vp, i32, i64, i32, i32, vp, vp, vp, vp, vp, i32, vp,
                                              ctypes.c_size_t, vp]
+    lib.skipffn_token_merge_scratch_bytes.restype = ctypes.c_size_t
+    lib.skipffn_token_merge_scratch_bytes.argtypes = [i64, i32, i32, i32]
+    lib.skipffn_token_merge.restype = i32
+    lib.skipffn_token_merge.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -177,6 +182,26 @@ def summary_backward(X, seg_offsets, w, probs, dxs, dw_fp32=False):
     if st != 0:
         raise SkipFFNError(st, "skipffn_summary_backward")
     return dX, dw
+
+
+def token_merge(X, k: int):
+    """Token merge of section 4.1 (``skipffn_token_merge``): ``(kept [k], assign [n], merged [k, C])``
+    for the tokens ``X [n, C]`` (bf16 or fp32 CUDA tensor)."""
+    import torch
+    lib = load_library()
+    dtype = BF16 if X.dtype == torch.bfloat16 else FP32
+    n, C = X.shape
+    kept = torch.empty(k, dtype=torch.int32, device=X.device)
+    assign = torch.empty(n, dtype=torch.int32, device=X.device)
+    merged = torch.empty(k, C, dtype=X.dtype, device=X.device)
+    nbytes = int(lib.skipffn_token_merge_scratch_bytes(n, C, k, dtype))
+    scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=X.device)
+    sp = (scratch.data_ptr() + 255) // 256 * 256
+    st = lib.skipffn_token_merge(_ptr(X), n, C, k, dtype, _ptr(kept), _ptr(assign), _ptr(merged),
+                                 ctypes.c_void_p(sp), nbytes, _stream_of(X))
+    if st != 0:
+        raise SkipFFNError(st, "skipffn_token_merge")
+    return kept, assign, merged
 
 
 def skipffn_compact_static(skip_mask, idx, nk) -> None:

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libskipffn.so")
-SOURCES = ["api.cu", "compact.cu", "compact_static.cu", "kvcache.cu", "prenorm.cu", "simt.cu", "summary.cu", "umma.cu"]
+SOURCES = ["api.cu", "compact.cu", "compact_static.cu", "kvcache.cu", "merge.cu", "prenorm.cu", "simt.cu", "summary.cu", "umma.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]
 

@@ -476,6 +476,25 @@ skipffn_status skipffn_summary_backward(const void *X, const int32_t *seg_offset
                                    (float *)scratch, (cudaStream_t)stream) == cudaSuccess ? SKIPFFN_OK : SKIPFFN_ECUDA;
 }
 
+size_t skipffn_token_merge_scratch_bytes(int64_t n, int32_t C, int32_t k, int32_t dtype)
+{
+    if (n <= 0 || C <= 0 || k <= 0 || k > n || (dtype != SKIPFFN_BF16 && dtype != SKIPFFN_FP32)) return 0;
+    return merge_scratch_bytes(n, C, k, dtype);
+}
+
+skipffn_status skipffn_token_merge(const void *X, int64_t n, int32_t C, int32_t k, int32_t dtype,
+                                   int32_t *kept, int32_t *assign, void *merged, void *scratch,
+                                   size_t scratch_bytes, void *stream)
+{
+    if (!X || !kept || !assign || !merged || !scratch || n <= 0 || k <= 0 || k > n || C <= 0) return SKIPFFN_EINVAL;
+    if (dtype != SKIPFFN_BF16 && dtype != SKIPFFN_FP32) return SKIPFFN_EINVAL;
+    if (C % 8 || C > 16384 || k % 4 || n > 65536) return SKIPFFN_EUNSUPPORTED;
+    if (!aligned16(X) || !aligned16(merged) || ((uintptr_t)scratch & 255u)) return SKIPFFN_EINVAL;
+    if (scratch_bytes < merge_scratch_bytes(n, C, k, dtype)) return SKIPFFN_EWORKSPACE;
+    return launch_token_merge(X, n, C, k, dtype, kept, assign, merged, scratch, (cudaStream_t)stream) == cudaSuccess
+               ? SKIPFFN_OK : SKIPFFN_ECUDA;
+}
+
 skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev, const int32_t **nk_dev)
 {
     if (!s || s->planned_N < 0) return SKIPFFN_EINVAL;

@@ -108,7 +108,9 @@ struct GemmArgs {
     int32_t sk_epoch;
 };
 
-enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_DX = 4 };
+// EPI_PLAIN: a plain GEMM with both operands K-major and the weight-gradient store (used by the
+// token-merge similarity matrix); the tensor-core path only.
+enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_DX = 4, EPI_PLAIN = 5 };
 
 // compact.cu
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
@@ -134,6 +136,10 @@ cudaError_t launch_summary_forward(const void *X, const int32_t *off, int n_seg,
 cudaError_t launch_summary_backward(const void *X, const int32_t *off, int n_seg, int64_t n, int C, int dtype,
                                     const void *w, const float *probs, const void *dxs, void *dX, void *dw,
                                     int dw_fp32, float *scratch, cudaStream_t s);
+// merge.cu
+size_t merge_scratch_bytes(int64_t n, int C, int k, int dtype);
+cudaError_t launch_token_merge(const void *X, int64_t n, int C, int k, int dtype, int32_t *kept, int32_t *assign,
+                               void *merged, void *scratch, cudaStream_t s);
 // simt.cu
 cudaError_t launch_simt_gemm(int epi, int dtype, const GemmArgs &a, cudaStream_t s);
 // umma.cu (bf16 only)

@@ -1009,6 +1009,7 @@ static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b,
     case EPI_DH:     return launch_k<EPI_DH, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
     case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
     case EPI_DX:     return launch_k<EPI_DX, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_PLAIN:  return launch_k<EPI_DW, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
     default: return cudaErrorInvalidValue;
     }
 }
@@ -1020,7 +1021,7 @@ static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b,
 // problems 1 and 2 share their B operand.
 static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStream_t s)
 {
-    if (n < 1 || n > 3 || (n > 1 && epi != EPI_DW)) return cudaErrorInvalidValue;
+    if (n < 1 || n > 3 || (n > 1 && epi != EPI_DW) || epi < 0 || epi > EPI_PLAIN) return cudaErrorInvalidValue;
     if (n == 3 && (gs[2].B != gs[1].B || gs[2].ldb_k != gs[1].ldb_k || gs[2].N != gs[1].N))
         return cudaErrorInvalidValue;
     if (g_num_sms == 0) {
@@ -1083,7 +1084,7 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_wait_skew = 0;
     if (const char *e = getenv("SKIPFFN_TEST_LOST_HANDOVER")) { if (atoi(e) != 0) p.sk_wait_skew = 0x40000000; }
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
-    static const int sk_threshold[5] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40};
+    static const int sk_threshold[6] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40, /*PLAIN*/ 32};
     p.streamk = (g.sk_slots && g.sk_flags) ? sk_threshold[epi] : 0;
     if (const char *e = getenv("SKIPFFN_STREAMK")) { int v = atoi(e); if (v >= 0) p.streamk = v; }
 
