@@ -476,6 +476,34 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // position in the SM pair; 0 leads
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int num_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    // ---- set-up that touches no global memory: barriers, tensor memory
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS * SPLIT);
+        }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        if (PAIR) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish_pair(); }
+        else      { tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish(); }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) cluster_sync_all();   // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    volatile int *abort_flag = &ctl->abort_flag;
+    // Programmatic dependent launch: the next kernel of the stream may start its own set-up while
+    // this one runs; everything below reads what earlier kernels wrote, so wait for them first.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int nk = p.status[ST_NK];
     const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
@@ -521,29 +549,6 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int b_slabs = (bn_cta + 63) / 64;
     const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
-        }
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS * SPLIT);
-        }
-        ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) {
-        if (PAIR) { tmem_alloc_pair(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish_pair(); }
-        else      { tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS); tmem_relinquish(); }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (PAIR) cluster_sync_all();   // the peer's barriers exist before anything signals them
-    tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
-    volatile int *abort_flag = &ctl->abort_flag;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -991,10 +996,16 @@ static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CU
     cfg.blockDim = dim3(UMMA_THREADS);
     cfg.dynamicSmemBytes = SMEM;
     cfg.stream = s;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = PAIR ? 2 : 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
+    // let this kernel's set-up overlap the tail of the previous kernel on the stream (the kernel
+    // itself waits for its predecessors before it reads global memory)
+    static int pdl = -1;
+    if (pdl < 0) { const char *e = getenv("SKIPFFN_PDL"); pdl = (e && atoi(e) == 0) ? 0 : 1; }
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kern, a, b, a2, b2, a3, p);
 }
 
