@@ -75,6 +75,27 @@ __device__ __forceinline__ void swiglu_bwd(float dh, float g, float u, float &dg
     dg = dh * u * (s * (1.0f + g * (1.0f - s)));
 }
 
+// Programmatic dependent launch.  Device side: let the next kernel of the stream start launching,
+// then wait until every earlier kernel has completed and its writes are visible (a no-op for a
+// kernel launched the ordinary way).  Must precede the kernel's first access to global memory.
+__device__ __forceinline__ void pdl_enter()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+// Host side: launch `kernel` so that its launch latency overlaps the tail of the previous kernel.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---------------------------------------------------------------- launch descriptors (host)
 struct RouteArgs {          // row routing: compact copy of kept rows + identity copy of skipped rows
     const void *src;        // [N, C]

@@ -24,6 +24,7 @@ k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__res
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned lt = (1u << lane) - 1u;
     int carry = 0;
+    pdl_enter();
     for (int64_t base = 0; base < N; base += (int64_t)CP_J * CP_THREADS) {
         unsigned bal[CP_J];
 #pragma unroll
@@ -78,8 +79,7 @@ k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__res
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
                            int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s)
 {
-    k_compact<<<1, CP_THREADS, 0, s>>>(mask, N, dense, idx, pos, status, cap);
-    return cudaGetLastError();
+    return launch_pdl(k_compact, dim3(1), dim3(CP_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
 }
 
 // Row routing.  Unit u < N is token u: a kept token's row goes to dst_compact[pos[u]], a skipped
@@ -94,6 +94,7 @@ k_route(const uint4 *__restrict__ src, uint4 *__restrict__ dst_compact,
         const int32_t *__restrict__ status, int64_t N, int row_vecs, int copy_identity)
 {
     int64_t u = blockIdx.x;
+    pdl_enter();
     if (u < N) {
         int p = pos[u];
         const uint4 *s = src + u * row_vecs;
@@ -126,10 +127,9 @@ cudaError_t launch_route(const RouteArgs &a, cudaStream_t s)
     int row_vecs = (int)((int64_t)a.C * a.elem_bytes / 16);
     int copy_identity = a.dst_identity != nullptr && a.dst_identity != a.src;
     int64_t units = a.N + ROW_PAD;
-    k_route<<<(unsigned)units, RT_THREADS, 0, s>>>(
-        (const uint4 *)a.src, (uint4 *)a.dst_compact, (uint4 *)a.dst_identity, a.pos, a.status,
-        a.N, row_vecs, copy_identity);
-    return cudaGetLastError();
+    return launch_pdl(k_route, dim3((unsigned)units), dim3(RT_THREADS), s, (const uint4 *)a.src,
+                      (uint4 *)a.dst_compact, (uint4 *)a.dst_identity, a.pos, a.status, a.N, row_vecs,
+                      copy_identity);
 }
 
 }  // namespace skipffn
