@@ -407,3 +407,10 @@ def test_bf16_gradient_accumulation():
         # one bf16 rounding of a value near |init|: absolute error below half an ulp of the sum
         assert np.max(np.abs(got - want)) <= 2.0 ** -8 * np.max(np.abs(want)) + 3e-2 * np.sqrt(np.mean(ref[k] ** 2))
         assert abs(np.mean(got - want)) < 1e-3
+
+
+def test_many_tokens_small_hidden():
+    # 40 000 tokens in 10 sequences (grids far beyond one wave of CTAs), narrow layer: full oracle
+    w = wl.uniform_batch(43, "bf16", 64, 128, 10, 100, 3800, 100, skip_ratio=0.9)
+    assert w.N == 40000 and w.n_kept == 10 * (200 + 380)
+    _compare(w, run(w), _oracle_all(w))
