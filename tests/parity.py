@@ -18,16 +18,13 @@ def rel_fro(got, ref):
     return num / den if den > 0 else num
 
 
-def row_maxabs_ratio(got, ref, floor_matrix_rms=False):
-    """max over rows of (max abs error of the row / RMS of the oracle row).  With
-    `floor_matrix_rms` a row's RMS is floored by the RMS of the whole matrix."""
+def row_maxabs_ratio(got, ref):
+    """max over rows of (max abs error of the row / RMS of the oracle row)."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     if ref.size == 0:
         return 0.0
     rms = np.sqrt(np.mean(ref * ref, axis=-1))
-    if floor_matrix_rms:
-        rms = np.maximum(rms, np.sqrt(np.mean(ref * ref)))
     err = np.max(np.abs(got - ref), axis=-1)
     ok = rms > 0
     ratio = np.zeros_like(err)
@@ -36,20 +33,56 @@ def row_maxabs_ratio(got, ref, floor_matrix_rms=False):
     return float(ratio.max())
 
 
-def check(got, ref, dtype, what, few_terms=False):
+BF16_UNIT_ROUNDOFF = 2.0 ** -8
+
+
+def few_term_dw_bounds(x_kept, dout_kept, W_gate, W_up, W_down):
+    """Elementwise first-order forward-error bounds for the three bf16 weight gradients when they
+    are sums over only a handful of kept tokens.
+
+    Why a separate criterion: a row of dW_gate summed over ONE token is dg[i] * x[t, :], so the
+    relative error of the single scalar dg[i] (which carries the bf16 roundings of the stored G, U
+    and dG) is shared by the whole row; the row's largest entry then misses the "3e-2 x row RMS"
+    criterion as soon as the row's peak-to-RMS ratio is large (heavy-tailed rows of dW_down do so
+    routinely), although every element is as accurate as bf16 storage allows.  With eight or more
+    terms the roundings are independent and the stated criterion holds; below that the elementwise
+    bound of the arithmetic itself is used instead:
+        dW_gate[i, c]: sum_t |x[t, c]| * |dh| * ( |u| |g silu''(g)| + 2 |u silu'(g)| ) * eps
+        dW_up  [i, c]: sum_t |x[t, c]| * |dh| * ( |g silu'(g)| + |silu(g)| ) * eps
+        dW_down[c, i]: sum_t |dout[t, c]| * |h| * eps
+    (eps = 2^-8, the unit roundoff of bf16: one term per rounding of G, U, dG / dU / H), plus
+    eps * |result| for the rounding of the output.  Inputs are the oracle's own float64 values."""
+    eps = BF16_UNIT_ROUNDOFF
+    x, do = np.asarray(x_kept, np.float64), np.asarray(dout_kept, np.float64)
+    wg, wu, wd = (np.asarray(a, np.float64) for a in (W_gate, W_up, W_down))
+    G, U, dH = x @ wg.T, x @ wu.T, do @ wd
+    S = 1.0 / (1.0 + np.exp(-G))
+    d1 = S * (1.0 + G * (1.0 - S))                         # silu'
+    d2 = S * (1.0 - S) * (2.0 + G * (1.0 - 2.0 * S))       # silu''
+    e_dg = np.abs(dH) * (np.abs(U) * np.abs(d2 * G) + 2.0 * np.abs(U * d1)) * eps
+    e_du = np.abs(dH) * (np.abs(d1 * G) + np.abs(G * S)) * eps
+    e_h = np.abs(G * S * U) * eps
+    return {"dW_gate": e_dg.T @ np.abs(x), "dW_up": e_du.T @ np.abs(x), "dW_down": np.abs(do).T @ e_h}
+
+
+def check(got, ref, dtype, what, elem_bound=None):
     """Assert the stated tolerance for `dtype` ('bf16' or 'fp32').
 
-    `few_terms`: the rows are sums over fewer than 8 kept tokens (weight gradients of a nearly
-    empty batch).  A row of dW_gate is then dg[i] * x[t] for a single token, and its relative
-    error is that of the one bf16 scalar dg[i], which is unbounded where silu'(g) crosses zero
-    because G is saved in bf16.  Those rows are tiny, so the per-row bound is taken against
-    max(row RMS, matrix RMS); the Frobenius bound is unchanged."""
+    `elem_bound` (bf16 weight gradients summed over fewer than 8 kept tokens only, see
+    few_term_dw_bounds): the per-row criterion is replaced by the elementwise bound
+    |error| <= 1.25 * (elem_bound + 2^-8 |ref|); the Frobenius criterion is unchanged."""
     assert np.all(np.isfinite(np.asarray(got, dtype=np.float64))), f"{what}: non-finite values"
     rf = rel_fro(got, ref)
     if dtype == "fp32":
         assert rf <= FP32_REL_FRO, f"{what}: rel Frobenius {rf:.3e} > {FP32_REL_FRO}"
     else:
         assert rf <= BF16_REL_FRO, f"{what}: rel Frobenius {rf:.3e} > {BF16_REL_FRO}"
-        rm = row_maxabs_ratio(got, ref, floor_matrix_rms=few_terms)
-        assert rm <= BF16_ROW_MAXABS, f"{what}: max abs / row RMS {rm:.3e} > {BF16_ROW_MAXABS}"
+        if elem_bound is not None:
+            err = np.abs(np.asarray(got, np.float64) - np.asarray(ref, np.float64))
+            lim = 1.25 * (elem_bound + BF16_UNIT_ROUNDOFF * np.abs(ref))
+            worst = float(np.max(err - lim))
+            assert worst <= 0.0, f"{what}: an element exceeds its forward-error bound by {worst:.3e}"
+        else:
+            rm = row_maxabs_ratio(got, ref)
+            assert rm <= BF16_ROW_MAXABS, f"{what}: max abs / row RMS {rm:.3e} > {BF16_ROW_MAXABS}"
     return rf

@@ -253,6 +253,65 @@ def test_sampled_modes_match_full():
     np.testing.assert_allclose(c, dwd[:, cols].T, rtol=1e-12, atol=1e-14)
 
 
+# ------------------------------------------------------------------ whole-matrix statement
+def _dense():
+    from oracle import dense
+    return dense
+
+
+@pytest.mark.parametrize("p_skip", [0.0, 0.5, 1.0])
+def test_dense_statement_equals_the_per_token_loops(p_skip):
+    # two statements of the same definition, written independently (C loops over tokens; numpy
+    # matmuls over the retained rows): they must agree to rounding on every result
+    x, mask, wg, wu, wd, dout = _rand_case(23, 10, 14, p_skip=p_skip, seed=61)
+    d = _dense().forward_backward(x, mask, wg, wu, wd, dout)
+    out = oracle.forward(x, mask, wg, wu, wd)
+    dx, dwg, dwu, dwd = oracle.backward(x, mask, wg, wu, wd, dout)
+    for got, want in ((d["out"], out), (d["dx"], dx), (d["dW_gate"], dwg), (d["dW_up"], dwu), (d["dW_down"], dwd)):
+        np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+    sk = mask != 0
+    assert d["out"][sk].tobytes() == x[sk].tobytes() and d["dx"][sk].tobytes() == dout[sk].tobytes()
+    if p_skip == 1.0:
+        assert not d["dW_gate"].any() and not d["dW_up"].any() and not d["dW_down"].any()
+
+
+def test_dense_statement_scalar_closed_form_and_finite_differences():
+    # C = I = 1: out = x + silu(x wg) (x wu) wd
+    r = _dense().forward_backward([[0.5]], [0], [[2.0]], [[-3.0]], [[0.25]])
+    z = 0.5 * 2.0
+    assert abs(r["out"][0, 0] - (0.5 + z / (1 + math.exp(-z)) * (0.5 * -3.0) * 0.25)) < 1e-15
+    # central differences of its own forward for the loss sum(dout * out)
+    x, mask, wg, wu, wd, dout = _rand_case(6, 4, 5, seed=71)
+    mask[0], mask[1] = 0, 1
+    d = _dense().forward_backward(x, mask, wg, wu, wd, dout)
+    loss = lambda *a: float(np.sum(dout * _dense().forward_backward(a[0], mask, a[1], a[2], a[3])["out"]))
+    args = [x, wg, wu, wd]
+    for k, name in enumerate(("dx", "dW_gate", "dW_up", "dW_down")):
+        num = np.zeros_like(args[k])
+        for pos in np.ndindex(*args[k].shape):
+            hi = [a.copy() for a in args]
+            lo = [a.copy() for a in args]
+            hi[k][pos] += 1e-6
+            lo[k][pos] -= 1e-6
+            num[pos] = (loss(*hi) - loss(*lo)) / 2e-6
+        np.testing.assert_allclose(d[name], num, rtol=1e-6, atol=1e-7)
+
+
+def test_dense_statement_prenorm_equals_the_per_token_loops():
+    x, mask, wg, wu, wd, dout = _rand_case(17, 12, 9, seed=81)
+    gamma = 1.0 + 0.2 * np.random.default_rng(3).normal(size=12)
+    d = _dense().forward_backward(x, mask, wg, wu, wd, dout, gamma=gamma, eps=1e-3)
+    out = oracle.forward_prenorm(x, mask, gamma, 1e-3, wg, wu, wd)
+    dx, dg, dwg, dwu, dwd = oracle.backward_prenorm(x, mask, gamma, 1e-3, wg, wu, wd, dout)
+    for got, want in ((d["out"], out), (d["dx"], dx), (d["dgamma"], dg), (d["dW_gate"], dwg), (d["dW_up"], dwu),
+                      (d["dW_down"], dwd)):
+        np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-12)
+    # a 3-4-0-0 row has mean square 6.25: with eps = 0 its normalised row is (1.2, 1.6, 0, 0)
+    one = _dense().forward_backward([[3.0, 4.0, 0.0, 0.0]], [0], np.eye(4), np.eye(4), np.eye(4), gamma=np.ones(4))
+    silu = lambda t: t / (1 + math.exp(-t))
+    np.testing.assert_allclose(one["out"][0], [3 + silu(1.2) * 1.2, 4 + silu(1.6) * 1.6, 0, 0], rtol=1e-14)
+
+
 # ------------------------------------------------------------------ paper closed forms
 def _golden():
     path = os.path.join(os.path.dirname(__file__), "golden", "llama3_8b_ffn_shape.txt")
