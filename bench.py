@@ -14,6 +14,15 @@ resident in HBM; `e2e` is the same metric with the step's inputs copied from pin
 and its results copied back inside the timed region; `roofline` describes the kernel with the
 largest share of the step; `cpu_baseline` is the fp64 CPU oracle timed on a bounded sample.
 With N > 1 (torchrun) every rank runs an independent replica (no collective on the data path).
+
+At N = 1 the same line carries, measured after and outside the headline timed region:
+  sustained  the same step repeated for at least 3 s: ms per step, TFLOP/s against the sustained
+             library peak, SM clock median and throttle reasons of that region, per-kernel times
+  cfg3/cfg4  the high-resolution and the packed variable-length workloads
+  sweep      skip ratios {0, .25, .5, .75, .9, 1} at both shapes against the in-library dense
+             comparator on the same inputs
+  host_us_per_step  host time of the eight launches of one step (no synchronisation)
+(`--no-extras` leaves them out.)
 """
 from __future__ import annotations
 
@@ -378,6 +387,48 @@ def run_ours(args):
                                          (sum(v["ms"] for v in gemms.values()) * 1e-3) / 1e12}}
         roofline["all_gemm_kernels"]["frac"] = roofline["all_gemm_kernels"]["tflops"] / pk["bf16_tflops"]
 
+    extras = {}
+    if world == 1 and not args.no_extras:
+        # host time of one step's launches: enqueue without synchronising
+        torch.cuda.synchronize()
+        th = time.perf_counter()
+        for _ in range(40):
+            step()
+        extras["host_us_per_step"] = (time.perf_counter() - th) / 40 * 1e6
+        torch.cuda.synchronize()
+        # sustained: the same step for at least 3 s, clocks sampled over that region
+        n_sus = max(args.steps, int(np.ceil(args.sustained_seconds * 1e3 / ms_step)))
+        sampler = ClockSampler(local)
+        ms_sus, t0, t1 = timed(step, n_sus)
+        clocks_sus = sampler.stop(t0, t1)
+        prof_sus = ctx.profile(step, 20)          # straight after, while the part is still power-capped
+        ctx.poll()
+        ms_s = ms_sus / n_sus
+        tf_s = sk.skipffn_flops(C, I, nk) / (ms_s * 1e-3) / 1e12
+        sus_kernels = {}
+        for name, kms in prof_sus.items():
+            ent = {"ms": kms}
+            if name in kernel_units:
+                ent["tflops"] = kernel_units[name] * unit_flops / (kms * 1e-3) / 1e12
+                if pk["bf16_tflops_sustained"]:
+                    ent["frac_of_sustained_bf16_peak"] = ent["tflops"] / pk["bf16_tflops_sustained"]
+            sus_kernels[name] = ent
+        extras["sustained"] = {
+            "steps": n_sus, "seconds": ms_sus * 1e-3, "ms_per_step": ms_s, "kept_tokens_per_s": nk / (ms_s * 1e-3),
+            "tflops": tf_s, "frac_of_sustained_bf16_peak": tf_s / pk["bf16_tflops_sustained"] if pk["bf16_tflops_sustained"] else None,
+            "frac_of_burst_bf16_peak": tf_s / pk["bf16_tflops"], "clocks": clocks_sus,
+            "mcycles_per_step": ms_s * clocks_sus["sm_mhz"] * 1e-3 if clocks_sus.get("sm_mhz") else None,
+            "kernels": sus_kernels}
+        # the other single-GPU workloads, same weights
+        dbuf.clear()
+        weights_host = (w.W_gate, w.W_up, w.W_down)
+        for name in ("cfg3", "cfg4"):
+            if args.workload == name or args.shape != "llama3-8b":
+                continue
+            wo = (wl.config3 if name == "cfg3" else wl.config4)(seed=args.seed, C=C, I=I, weights=weights_host)
+            extras[name] = time_workload(sk, wo, (Wg, Wu, Wd), (dWg, dWu, dWd), args.steps, max(args.warmup, 3), pk)
+        extras["sweep"] = sweep_table(sk, args, pk, {args.shape: (Wg, Wu, Wd)})
+
     cpu = None
     if not args.no_cpu_baseline and world == 1:    # the oracle is timed at N = 1 only
         rate, kept, dt, cores = oracle_sample_rate(w, args.cpu_sample_tokens)
@@ -392,78 +443,113 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config(args, w), "tflops": tflops,
             "frac_of_measured_bf16_peak": tflops / world / pk["bf16_tflops"],
-            "frac_of_sustained_bf16_peak": (tflops / world / pk["bf16_tflops_sustained"]) if pk["bf16_tflops_sustained"] else None,
             "frac_of_nominal_bf16_peak": tflops / world / 2250.0,
+            "timed_region": "burst: %d steps, %.0f ms; see `sustained` for the power-capped figure" % (args.steps, ms_step * args.steps),
             "e2e": {"value": value_e2e, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_step_e2e,
                     "pipeline": "3 streams (H2D, compute, D2H), double-buffered device inputs and results"},
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
             "kernels": kernels, "cpu_baseline": cpu}
+    line.update(extras)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------ other workloads
+def _h_bf16(a):
+    import torch
+    return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).reshape(a.shape)
+
+
+def time_ctx(ctx, x, mask, dout, W, bufs, steps, warmup):
+    """ms per forward+backward step of `ctx` on resident inputs (CUDA events, after warm-up)."""
+    import torch
+    out, dx, dWg, dWu, dWd = bufs
+
+    def step():
+        ctx.forward(x, mask, W[0], W[1], W[2], out=out)
+        ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+    for _ in range(max(warmup, 3)):
+        step()
+    ctx.poll()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ctx.poll()
+    return e0.elapsed_time(e1) / steps
+
+
+def time_workload(sk, w, W, dW, steps, warmup, pk):
+    """One more workload on weights already on the device: ms per step, kept tokens/s, TFLOP/s."""
+    import torch
+    x, dout, mask = _h_bf16(w.x).cuda(), _h_bf16(w.dout).cuda(), torch.from_numpy(w.skip_mask).cuda()
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    ms = time_ctx(ctx, x, mask, dout, W, [torch.empty_like(x), torch.empty_like(x)] + list(dW), steps, warmup)
+    tf = sk.skipffn_flops(w.C, w.I, w.n_kept) / (ms * 1e-3) / 1e12
+    return {"workload": w.name, "tokens": w.N, "kept_tokens": w.n_kept, "steps": steps, "ms_per_step": ms,
+            "kept_tokens_per_s": w.n_kept / (ms * 1e-3), "tflops": tf,
+            "frac_of_measured_bf16_peak": tf / pk["bf16_tflops"]}
+
+
 # ------------------------------------------------------------------------------ skip-ratio sweep
-def run_sweep(args):
+def sweep_table(sk, args, pk, resident=None):
     """Skip-ratio sweep: visual skip fraction in {0, .25, .5, .75, .9, 1} at the LLaMA3-8B and
     Vicuna-13B shapes (8 x 616 tokens), plus the in-library dense comparator on the same inputs.
-    One JSON line: per point kept tokens/s, TFLOP/s and time relative to dense."""
+    Per point: kept tokens/s, TFLOP/s, time relative to dense, and the floor that time is held
+    against: max(kept fraction, time to stream the weights and write the weight gradients once at
+    the measured HBM rate / dense time).  `resident`: weights of a shape already on the device."""
     import torch
-    import paper_2503_21817_b200 as sk
-    torch.cuda.set_device(0)
-    pk = peaks()
-
-    def h_bf16(a):
-        return torch.from_numpy(wl.to_bf16_bits(a).view(np.int16)).view(torch.bfloat16).reshape(a.shape)
-
-    def time_ctx(ctx, x, mask, dout, W, bufs):
-        out, dx, dWg, dWu, dWd = bufs
-
-        def step():
-            ctx.forward(x, mask, W[0], W[1], W[2], out=out)
-            ctx.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
-        for _ in range(max(args.warmup, 3)):
-            step()
-        ctx.poll()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(args.steps):
-            step()
-        e1.record()
-        torch.cuda.synchronize()
-        ctx.poll()
-        return e0.elapsed_time(e1) / args.steps
-
     table = {}
     for shape, (C, I) in wl.SWEEP_SHAPES.items():
-        base = wl.config2(seed=args.seed, skip_ratio=0.0, C=C, I=I)
-        weights = (base.W_gate, base.W_up, base.W_down)
-        W = [h_bf16(a).cuda() for a in weights]
-        x, dout = h_bf16(base.x).cuda(), h_bf16(base.dout).cuda()
+        if resident and shape in resident:
+            W = list(resident[shape])
+            base = wl.config2(seed=args.seed, skip_ratio=0.0, C=C, I=I,
+                              weights=tuple(np.empty((0,), np.float32) for _ in range(3)))
+        else:
+            base = wl.config2(seed=args.seed, skip_ratio=0.0, C=C, I=I)
+            W = [_h_bf16(a).cuda() for a in (base.W_gate, base.W_up, base.W_down)]
+        x, dout = _h_bf16(base.x).cuda(), _h_bf16(base.dout).cuda()
         bufs = [torch.empty_like(x), torch.empty_like(x)] + [torch.empty_like(t) for t in W]
         dense = sk.SkipFFN(C, I, base.N, dense=True)
-        ms_dense = time_ctx(dense, x, torch.from_numpy(base.skip_mask).cuda(), dout, W, bufs)
+        ms_dense = time_ctx(dense, x, torch.from_numpy(base.skip_mask).cuda(), dout, W, bufs, args.steps, args.warmup)
         del dense
         ctx = sk.SkipFFN(C, I, base.N)
+        # weights read by forward and backward, weight gradients written: 9 C I bf16 elements
+        ms_weights = 9.0 * C * I * 2 / (pk["hbm_gbs"] * 1e9) * 1e3
         rows = []
         for r in wl.SWEEP_RATIOS:
             m = wl.config2(seed=args.seed, skip_ratio=r, C=8, I=8).skip_mask   # the mask depends on (seed, r) only
             nk = int((m == 0).sum())
-            ms = time_ctx(ctx, x, torch.from_numpy(m).cuda(), dout, W, bufs)
+            ms = time_ctx(ctx, x, torch.from_numpy(m).cuda(), dout, W, bufs, args.steps, args.warmup)
             tf = sk.skipffn_flops(C, I, nk) / (ms * 1e-3) / 1e12
+            floor = max(nk / base.N, ms_weights / ms_dense)
             rows.append({"skip_ratio": r, "kept_tokens": nk, "ms_per_step": ms, "kept_tokens_per_s": nk / (ms * 1e-3),
                          "tflops": tf, "frac_of_measured_bf16_peak": tf / pk["bf16_tflops"],
-                         "time_vs_dense": ms / ms_dense, "kept_fraction": nk / base.N})
+                         "time_vs_dense": ms / ms_dense, "kept_fraction": nk / base.N,
+                         "floor": floor, "time_vs_dense_over_floor": ms / ms_dense / floor})
         tf_dense = sk.skipffn_flops(C, I, base.N) / (ms_dense * 1e-3) / 1e12
-        table[shape] = {"C": C, "I": I, "tokens": base.N,
+        table[shape] = {"C": C, "I": I, "tokens": base.N, "weight_streaming_floor_ms": ms_weights,
                         "dense": {"ms_per_step": ms_dense, "tflops": tf_dense,
                                   "frac_of_measured_bf16_peak": tf_dense / pk["bf16_tflops"]},
                         "points": rows}
         del ctx, W, x, dout, bufs
+    return table
+
+
+def run_sweep(args):
+    """The sweep alone, as one JSON line."""
+    import torch
+    import paper_2503_21817_b200 as sk
+    torch.cuda.set_device(0)
+    pk = peaks()
     print(json.dumps({"sweep": "skip ratio", "steps": args.steps, "dtype": "bf16", "data": "synthetic",
-                      "peak_tflops": pk["bf16_tflops"], "peak_source": pk["source"], "shapes": table}), flush=True)
+                      "peak_tflops": pk["bf16_tflops"], "peak_source": pk["source"],
+                      "shapes": sweep_table(sk, args, pk)}), flush=True)
 
 
 # ------------------------------------------------------------------------------ skip KV-cache
@@ -659,6 +745,9 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="leave out the sustained / cfg3 / cfg4 / sweep keys (N = 1 only carries them)")
+    ap.add_argument("--sustained-seconds", type=float, default=3.0)
     ap.add_argument("--profile-only", action="store_true",
                     help="run warmup+steps steps and exit (launch sequence for an ncu capture)")
     ap.add_argument("--sweep", action="store_true",

@@ -212,7 +212,7 @@ def skipffn_compact_static(skip_mask, idx, nk) -> None:
     int32 with one entry.  Neither this wrapper nor the library call allocates anything; the
     kernel's scratch is a fixed array inside the library, which limits N to ``STATIC_MAX_TOKENS``
     and means that calls overlapping on the GPU must be serialised by the caller.  Enqueued on the
-    current torch stream."""
+    current torch stream of the tensors' GPU, which is made current for the call."""
     import torch
     N = skip_mask.numel()
     if skip_mask.dtype != torch.uint8 or idx.dtype != torch.int32 or nk.dtype != torch.int32:
@@ -220,8 +220,12 @@ def skipffn_compact_static(skip_mask, idx, nk) -> None:
     if not (skip_mask.is_cuda and idx.is_cuda and nk.is_cuda and skip_mask.is_contiguous()
             and idx.is_contiguous()) or idx.numel() < N or nk.numel() < 1:
         raise ValueError("skip_mask, idx (>= N entries) and nk (1 entry) must be contiguous CUDA tensors")
-    stream = ctypes.c_void_p(torch.cuda.current_stream(skip_mask.device).cuda_stream)
-    st = load_library().skipffn_compact_static(_ptr(skip_mask), N, _ptr(idx), _ptr(nk), stream)
+    if idx.device != skip_mask.device or nk.device != skip_mask.device:
+        raise ValueError("skip_mask, idx and nk must live on the same GPU")
+    # the library resolves its fixed array for the CURRENT device, so make the tensors' GPU current
+    with torch.cuda.device(skip_mask.device):
+        stream = ctypes.c_void_p(torch.cuda.current_stream(skip_mask.device).cuda_stream)
+        st = load_library().skipffn_compact_static(_ptr(skip_mask), N, _ptr(idx), _ptr(nk), stream)
     if st == 2:
         raise SkipFFNError(st, f"skipffn_compact_static: N = {N} exceeds the fixed scratch of "
                                f"{STATIC_MAX_TOKENS} tokens")

@@ -4,9 +4,10 @@ The entry point keeps the compaction kernel's scratch in a fixed array inside th
 of a caller-allocated workspace, so it serves code that must not (or cannot) call cudaMalloc: a
 process whose framework already owns all device memory, a loop that cannot take cudaMalloc's
 device-wide synchronisation, a host that forbids allocation from extensions.  Here it is called
-through the C ABI twice in a row on different masks (the second shorter, so stale scratch from
-the first call would show) and compared bit for bit with the list the regular handle-based entry
-point (skipffn_plan + skipffn_get_kept) produces.  Collected last on purpose."""
+through the C ABI twice in a row on different masks and compared bit for bit with the list the
+regular handle-based entry point (skipffn_plan + skipffn_get_kept) produces.  The second mask is
+shorter and keeps other tokens, so a kept count or a rank left over from the first call (both live
+in the shared array) would give a wrong length or wrong entries.  Collected last on purpose."""
 import ctypes
 
 import numpy as np
