@@ -248,6 +248,8 @@ def run_ours(args):
     out, dx = torch.empty_like(x), torch.empty_like(x)
     dWg, dWu, dWd = torch.empty_like(Wg), torch.empty_like(Wu), torch.empty_like(Wd)
     ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense, prenorm=args.prenorm)
+    if args.tune:       # launch knobs of the handle (skipffn_tune), e.g. --tune one_box=0,streamk=0
+        ctx.tune(**{k: int(v) for k, v in (kv.split("=") for kv in args.tune.split(","))})
     if args.dense:
         nk = N
     fwd_kw, bwd_kw = {}, {}
@@ -745,6 +747,7 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tune", default="", help="comma-separated skipffn_tune knobs for the headline context, e.g. one_box=0")
     ap.add_argument("--no-extras", action="store_true",
                     help="leave out the sustained / cfg3 / cfg4 / sweep keys (N = 1 only carries them)")
     ap.add_argument("--sustained-seconds", type=float, default=3.0)

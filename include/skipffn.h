@@ -57,6 +57,7 @@ typedef struct {
     int32_t accumulate_dw;   /* 1: dW += ..., 0: dW is overwritten */
     int32_t path;            /* skipffn_path */
     int32_t prenorm;         /* 1: pre-norm variant (skipffn_forward_prenorm / _backward_prenorm) */
+    int32_t debug;           /* 1: debug handle: extra device-side checks (see skipffn_poll), test hooks */
 } skipffn_config;
 
 /* Host-side handle linking one forward call to its backward call.  It points into the caller's
@@ -72,6 +73,25 @@ size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens);
 skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg,
                                     void *workspace, size_t workspace_bytes, int64_t max_tokens);
 void skipffn_saved_destroy(skipffn_saved *saved);
+
+/* Tuning and test knobs of a handle (host-only; none is needed in normal use).  They affect the
+ * tensor-core GEMM launches that follow.
+ *   TILE_N          accumulator columns per tile instead of 256: a multiple of 16 (token problems)
+ *                   or 32 (weight gradients) in 32 .. 256; 0 = default
+ *   STREAMK         least number of K-blocks per worker that cutting the tail tiles along K must
+ *                   save for the cut to be used: 0 never cut, 1 cut whenever the tiles do not fill
+ *                   a wave, -1 = default per kernel
+ *   STAGES          use only this many stages of the shared-memory ring (1 .. 5); 0 = all
+ *   ONE_BOX         1 (default): an operand tile that consists of two 64-wide pieces (the two slabs
+ *                   of a transposed operand; the gate and the up rows) is fetched with one 3-D
+ *                   TMA box where the arrays allow it; 0: always one 2-D box per piece
+ *   LOSE_HANDOVER   debug handles only (EINVAL otherwise): nonzero makes the finishing units of a
+ *                   K-split launch wait for a hand-over that never comes, so that the bounded wait
+ *                   runs out and skipffn_poll reports SKIPFFN_ETIMEOUT -- the failure path can be
+ *                   exercised without any fault */
+typedef enum { SKIPFFN_TUNE_TILE_N = 0, SKIPFFN_TUNE_STREAMK = 1, SKIPFFN_TUNE_STAGES = 2,
+               SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_COUNT = 5 } skipffn_tunable;
+skipffn_status skipffn_tune(skipffn_saved *saved, int32_t what, int32_t value);
 
 /* Mask compaction alone (the retained / skipped split is the same for every decoder layer, so a
  * caller may build it once): writes the ascending kept-row index list and its length into the
@@ -182,7 +202,8 @@ skipffn_status skipffn_kv_compact(const skipffn_saved *saved, const void *src, v
                                   int32_t *kept_cu_seqlens, void *stream);
 
 /* Device addresses of the compacted intermediates of the last forward / backward, each
- * [round_up(Nk,128), I] in cfg.dtype (rows >= Nk are zero): which = 0 G, 1 U, 2 H, 3 dG, 4 dU;
+ * [Nk, I] in cfg.dtype (rows Nk .. round_up(Nk,16)-1 are zero, later rows are unspecified):
+ * which = 0 G, 1 U, 2 H, 3 dG, 4 dU;
  * 5 = kept rows of x [.., C]; 6 = kept rows of dout [.., C]; 7 = normalised kept rows of x
  * [.., C] (pre-norm variant only). */
 skipffn_status skipffn_get_intermediate(const skipffn_saved *saved, int32_t which,

@@ -20,9 +20,10 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact",
            "skipffn_forward_prenorm", "skipffn_backward_prenorm", "skipffn_summary_scratch_bytes",
            "skipffn_summary_forward", "skipffn_summary_backward", "skipffn_token_merge_scratch_bytes",
-           "skipffn_token_merge"]
+           "skipffn_token_merge", "skipffn_tune"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
+TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4}
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
                  "dw_up", "dx", "norm_bwd"]
 
@@ -37,7 +38,7 @@ class _Config(ctypes.Structure):
     _fields_ = [("C", ctypes.c_int32), ("I", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("dense", ctypes.c_int32), ("grad_dtype_fp32", ctypes.c_int32),
                 ("accumulate_dw", ctypes.c_int32), ("path", ctypes.c_int32),
-                ("prenorm", ctypes.c_int32)]
+                ("prenorm", ctypes.c_int32), ("debug", ctypes.c_int32)]
 
 
 def load_library() -> ctypes.CDLL:
@@ -59,6 +60,8 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_saved_destroy.argtypes = [vp]
     lib.skipffn_plan.restype = i32
     lib.skipffn_plan.argtypes = [vp, vp, i64, vp]
+    lib.skipffn_tune.restype = i32
+    lib.skipffn_tune.argtypes = [vp, i32, i32]
     lib.skipffn_forward.restype = i32
     lib.skipffn_forward.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp, vp, vp]
     lib.skipffn_backward.restype = i32
@@ -105,9 +108,9 @@ def load_library() -> ctypes.CDLL:
 
 
 def _cfg(C, I, dtype=BF16, dense=False, grad_fp32=False, accumulate_dw=False, path=PATH_DEFAULT,
-         prenorm=False):
+         prenorm=False, debug=False):
     return _Config(int(C), int(I), int(dtype), int(bool(dense)), int(bool(grad_fp32)),
-                   int(bool(accumulate_dw)), int(path), int(bool(prenorm)))
+                   int(bool(accumulate_dw)), int(path), int(bool(prenorm)), int(bool(debug)))
 
 
 def skipffn_workspace_bytes(C, I, max_tokens, dtype=BF16) -> int:
@@ -243,7 +246,7 @@ class SkipFFN:
 
     def __init__(self, C: int, I: int, max_tokens: int, dtype: int = BF16, dense: bool = False,
                  grad_fp32: bool = False, accumulate_dw: bool = False, path: int = PATH_DEFAULT,
-                 device="cuda", prenorm: bool = False):
+                 device="cuda", prenorm: bool = False, debug: bool = False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("Skip-FFN needs a CUDA device (sm_100a); there is no CPU path")
@@ -252,7 +255,7 @@ class SkipFFN:
         self.C, self.I, self.dtype, self.max_tokens = int(C), int(I), int(dtype), int(max_tokens)
         self.grad_fp32 = bool(grad_fp32) or dtype == FP32
         self.prenorm = bool(prenorm)
-        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path, prenorm)
+        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path, prenorm, debug)
         self.device = torch.device(device)
         nbytes = int(self.lib.skipffn_workspace_bytes(ctypes.byref(self.cfg), self.max_tokens))
         if nbytes == 0:
@@ -292,6 +295,13 @@ class SkipFFN:
             raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
 
     # ------------------------------------------------------------------ C-ABI mirrors
+    def tune(self, **knobs):
+        """``skipffn_tune``: tile_n, streamk, stages, lose_handover (debug contexts only)."""
+        for name, value in knobs.items():
+            st = self.lib.skipffn_tune(self._saved, TUNABLES[name], int(value))
+            if st != 0:
+                raise SkipFFNError(st, f"skipffn_tune({name})")
+
     def plan(self, skip_mask):
         self._check(skip_mask, "skip_mask", dtype=self._torch.uint8)
         st = self.lib.skipffn_plan(self._saved, _ptr(skip_mask), skip_mask.numel(), self._stream())

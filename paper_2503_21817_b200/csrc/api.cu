@@ -25,6 +25,8 @@ struct skipffn_saved {
     const void *Wg, *Wu, *Wd;
     int launches[2];
     int32_t sk_epoch;      // flag value of the latest tensor-core GEMM launch (never 0)
+    int32_t tune[SKIPFFN_TUNE_COUNT];   // skipffn_tune values
+    TmapCache tmaps;       // encoded tensor maps of the arrays this handle launches on
     // optional per-launch timing (CUDA events on the caller's stream)
     int profiling;
     cudaEvent_t ev[2 * SKIPFFN_PROFILE_SLOTS];
@@ -41,7 +43,7 @@ bool valid_cfg(const skipffn_config *c)
 {
     return c && c->C > 0 && c->I > 0 && (c->dtype == SKIPFFN_BF16 || c->dtype == SKIPFFN_FP32) &&
            (c->path == SKIPFFN_PATH_DEFAULT || c->path == SKIPFFN_PATH_SIMT) &&
-           (c->prenorm == 0 || c->prenorm == 1);
+           (c->prenorm == 0 || c->prenorm == 1) && (c->debug == 0 || c->debug == 1);
 }
 
 Layout make_layout(const skipffn_config *c, int64_t max_tokens)
@@ -106,7 +108,7 @@ cudaError_t run_gemm(skipffn_saved *s, int slot, int epi, GemmArgs &g, cudaStrea
     });
 }
 
-GemmArgs base_args(const skipffn_saved *s)
+GemmArgs base_args(skipffn_saved *s)
 {
     GemmArgs g;
     memset(&g, 0, sizeof(g));
@@ -114,6 +116,14 @@ GemmArgs base_args(const skipffn_saved *s)
     g.idx = s->idx;
     g.sk_slots = s->sk_slots;
     g.sk_flags = s->sk_flags;
+    g.tune_tile_n = s->tune[SKIPFFN_TUNE_TILE_N];
+    g.tune_stages = s->tune[SKIPFFN_TUNE_STAGES];
+    g.tune_streamk = s->tune[SKIPFFN_TUNE_STREAMK];
+    // failure-path hook of debug handles: finishing units of a K-split launch wait for a hand-over
+    // flag value that nothing writes, so their bounded wait runs out
+    g.sk_wait_skew = (s->cfg.debug && s->tune[SKIPFFN_TUNE_LOSE_HANDOVER]) ? 0x40000000 : 0;
+    g.one_box_loads = s->tune[SKIPFFN_TUNE_ONE_BOX];
+    g.tmaps = &s->tmaps;
     return g;
 }
 
@@ -172,7 +182,17 @@ skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config 
     s->Xn = w + l.Xn; s->rstd = (float *)(w + l.rstd); s->dY = (float *)(w + l.dY);
     s->dg_part = (float *)(w + l.dg_part);
     s->planned_N = -1;
+    s->tune[SKIPFFN_TUNE_STREAMK] = -1;
+    s->tune[SKIPFFN_TUNE_ONE_BOX] = 1;
     *saved = s;
+    return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_tune(skipffn_saved *s, int32_t what, int32_t value)
+{
+    if (!s || what < 0 || what >= SKIPFFN_TUNE_COUNT) return SKIPFFN_EINVAL;
+    if (what == SKIPFFN_TUNE_LOSE_HANDOVER && !s->cfg.debug) return SKIPFFN_EINVAL;
+    s->tune[what] = value;
     return SKIPFFN_OK;
 }
 
@@ -271,19 +291,35 @@ static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_
         }) != cudaSuccess)
         return SKIPFFN_ECUDA;
 
-    // G = A Wg^T, U = A Wu^T, H = silu(G) * U, with A = the kept rows (normalised in the pre-norm variant)
+    // G = X Wg^T, U = X Wu^T, H = silu(G) * U, with X = the kept rows (normalised in the pre-norm
+    // variant).  The tensor-core kernels take the weights as the A operand (weight rows along the
+    // accumulator rows) and the token rows as B; the plain-FMA kernels the other way round.
+    const void *Xrows = gamma ? s->Xn : s->Xk;
+    const bool tc = use_umma(s);
     GemmArgs g = base_args(s);
-    g.A = gamma ? s->Xn : s->Xk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
-    g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
-    g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+    if (tc) {
+        g.A = W_gate; g.A2 = W_up; g.lda_m = C; g.lda_k = 1; g.a_outer = I;
+        g.B = Xrows; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap;
+        g.M = I; g.N = (int32_t)N; g.n_from_nk = 1; g.K = C;
+    } else {
+        g.A = Xrows; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+        g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
+        g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+    }
     g.out0 = s->G; g.out1 = s->U; g.out2 = s->H; g.ldo = I;
     if (run_gemm(s, SLOT_GATEUP, EPI_GATEUP, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
 
     // out[idx[r]] = Xk[r] + H Wd^T
     g = base_args(s);
-    g.A = s->H; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
-    g.B = W_down; g.ldb_n = I; g.ldb_k = 1; g.b_outer = C;
-    g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+    if (tc) {
+        g.A = W_down; g.lda_m = I; g.lda_k = 1; g.a_outer = C;
+        g.B = s->H; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap;
+        g.M = C; g.N = (int32_t)N; g.n_from_nk = 1; g.K = I;
+    } else {
+        g.A = s->H; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+        g.B = W_down; g.ldb_n = I; g.ldb_k = 1; g.b_outer = C;
+        g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+    }
     g.in0 = s->Xk; g.out0 = out; g.ldo = C;
     if (run_gemm(s, SLOT_DOWN, EPI_DOWN, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     s->forwarded = 1;
@@ -322,6 +358,7 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
     const int C = s->cfg.C, I = s->cfg.I;
     s->launches[1] = 0;
     GemmArgs g;
+    const bool tc = use_umma(s);
 
     if (N > 0) {
         RouteArgs r;
@@ -332,9 +369,15 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
 
         // dH = dOk Wd ; dG, dU through the activation
         g = base_args(s);
-        g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
-        g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;
-        g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+        if (tc) {   // dH^T[i, t] = sum_c Wd[c, i] dOk[t, c]
+            g.A = s->Wd; g.lda_m = 1; g.lda_k = I; g.a_outer = C;
+            g.B = s->dOk; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap;
+            g.M = I; g.N = (int32_t)N; g.n_from_nk = 1; g.K = C;
+        } else {
+            g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+            g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;
+            g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+        }
         g.in0 = s->G; g.in1 = s->U; g.out0 = s->dG; g.out1 = s->dU; g.ldo = I;
         if (run_gemm(s, SLOT_DH, EPI_DH, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
     } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
@@ -377,9 +420,15 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
 
     if (N > 0) {   // dx[idx[r]] = dOk[r] + dG Wg + dU Wu
         g = base_args(s);
-        g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
-        g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
-        g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+        if (tc) {   // dx^T[c, t] = sum_i Wg[i, c] dG[t, i] + Wu[i, c] dU[t, i]
+            g.A = s->Wg; g.A2 = s->Wu; g.lda_m = 1; g.lda_k = C; g.a_outer = I;
+            g.B = s->dG; g.B2 = s->dU; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap;
+            g.M = C; g.N = (int32_t)N; g.n_from_nk = 1; g.K = I;
+        } else {
+            g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+            g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
+            g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+        }
         if (prenorm) { g.in0 = nullptr; g.out0 = s->dY; g.out_fp32 = 1; }   // gradient w.r.t. the normalised rows
         else { g.in0 = s->dOk; g.out0 = dx; }
         g.ldo = C;

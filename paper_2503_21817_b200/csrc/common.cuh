@@ -11,11 +11,11 @@ namespace skipffn {
 typedef __nv_bfloat16 bf16;
 
 // Device status block at the start of the workspace (int32 words).
-enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_WORDS = 64 };
+enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_ROLE_BASE = 16, ST_WORDS = 64 };   // ST_ROLE_BASE..: optional role cycle counters
 
 // Wait sites reported through the status word when a bounded wait gives up.
 enum : int { SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_TMEM_EMPTY = 3,
-             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6 };
+             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6, SITE_EPI_EXCHANGE = 7 };
 
 // Split-K hand-over between CTAs of one tensor-core GEMM launch: a CTA that computes only part
 // of a tile's K range leaves its fp32 accumulator in its own slot of the workspace and raises one
@@ -108,13 +108,23 @@ struct RouteArgs {          // row routing: compact copy of kept rows + identity
     int32_t elem_bytes;
 };
 
+// Encoded TMA tensor maps of the arrays a handle keeps seeing (weights, workspace slabs, the
+// caller's activations); lives in the handle, filled and searched by the launch code.
+constexpr int TMAP_BYTES = 128, TMAP_CACHE_ENTRIES = 48;
+struct TmapKey { const void *base; int64_t inner, outer, pitch; int box_outer; int64_t dim2, stride2; };
+struct TmapCache {
+    int used, next;
+    TmapKey key[TMAP_CACHE_ENTRIES];
+    alignas(64) unsigned char map[TMAP_CACHE_ENTRIES][TMAP_BYTES];
+};
+
 struct GemmArgs {
-    // C[m, n] = sum_k A(m, k) * B(n, k)  (+ second segment A2/B2 when K2 > 0)
+    // C[m, n] = sum_k A(m, k) * B(n, k)  (+ second segment A2/B2 for dX)
     const void *A, *B, *A2, *B2;
     int64_t lda_m, lda_k, ldb_n, ldb_k;
     int64_t a_outer, b_outer;   // addressable rows of the A / B arrays (tensor-map extents)
-    int32_t M, N, K;            // host upper bounds; *_dev overrides when >= 0
-    int32_t m_from_nk, k_from_nk;   // 1: the extent is the device-resident kept count
+    int32_t M, N, K;            // host upper bounds
+    int32_t m_from_nk, n_from_nk, k_from_nk;   // 1: the extent is the device-resident kept count
     const int32_t *status;      // status block
     const int32_t *idx;         // kept-row list for scatter epilogues
     // epilogue operands
@@ -127,6 +137,11 @@ struct GemmArgs {
     void *sk_slots;
     int32_t *sk_flags;
     int32_t sk_epoch;
+    int32_t sk_wait_skew;       // 0; debug handles: make finishing units wait for a value nobody writes
+    // tensor-core path: tuning overrides of the handle (0 / -1 = defaults) and its tensor-map cache
+    int32_t tune_tile_n, tune_stages, tune_streamk;
+    int32_t one_box_loads;      // 1: load an operand tile with one 3-D box where the arrays allow it
+    TmapCache *tmaps;
 };
 
 // EPI_PLAIN: a plain GEMM with both operands K-major and the weight-gradient store (used by the

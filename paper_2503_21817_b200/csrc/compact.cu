@@ -4,20 +4,113 @@
 
 namespace skipffn {
 
-// One CTA of 1024 threads walks the mask in slabs of 16 x 1024 tokens.  Within a slab, token
-// (j, warp, lane) = base + j*1024 + warp*32 + lane; a warp ballot gives each kept token its rank
-// inside its 32-token segment, and an exclusive scan over the 512 segment counts (segments are in
-// ascending token order) gives the segment's offset.  The list is therefore ascending (stable).
+// Mask compaction.  Outputs (all ascending, i.e. a stable compaction):
 //   idx[r]  : token index of the r-th kept token, r < Nk; entries Nk .. round_up(Nk, ROW_PAD)-1
-//             repeat a valid kept token (or 0) so that padded gathers stay in bounds
+//             (inside idx's capacity) are 0, a valid row, so that padded gathers stay in bounds
 //   pos[t]  : rank of token t among kept tokens, or -1 if skipped
 //   status[ST_NK] = Nk
+//
+// k_compact: one CTA per block of 4096 tokens, no communication between CTAs.  A CTA first counts
+// the kept tokens in front of its block by reading that part of the mask itself (at most N bytes,
+// from L2 after the first CTA touched them), then ranks its own 4096 tokens: every thread owns 16
+// consecutive tokens, a ballot-free bit count gives its share, a two-level shuffle scan its offset.
+// The last CTA also knows the total and writes Nk and the padding entries.  The redundant counting
+// grows with N^2 / 8192 bytes, so very long inputs take the single-CTA kernel below instead.
+constexpr int CB_THREADS = 256;
+constexpr int CB_PER_THREAD = 16;
+constexpr int CB_TOKENS = CB_THREADS * CB_PER_THREAD;      // 4096 tokens per CTA
+constexpr int64_t CB_MAX_N = 262144;                        // beyond: k_compact_serial
+
+// number of kept tokens among bytes [lo, hi) of the mask, summed over the CTA (valid in every thread)
+__device__ __forceinline__ int block_sum(int v, int *warp_tot)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    if (lane == 0) warp_tot[warp] = v;
+    __syncthreads();
+    int t = 0;
+#pragma unroll
+    for (int w = 0; w < CB_THREADS / 32; ++w) t += warp_tot[w];
+    __syncthreads();
+    return t;
+}
+
+__global__ void __launch_bounds__(CB_THREADS)
+k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
+          int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
+{
+    __shared__ int warp_tot[CB_THREADS / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t base = (int64_t)blockIdx.x * CB_TOKENS;
+    pdl_enter();
+    // ---- kept tokens in front of this block
+    int before = 0;
+    if (dense) {
+        before = (int)base;
+    } else {
+        int cnt = 0;
+        const bool vec = (((uintptr_t)mask) & 15u) == 0;
+        if (vec) {
+            const uint4 *m4 = reinterpret_cast<const uint4 *>(mask);
+            for (int64_t v = tid; v < base / 16; v += CB_THREADS) {   // base is a multiple of 16
+                const uint4 q = __ldg(m4 + v);
+                cnt += (__popc(__vcmpeq4(q.x, 0u)) + __popc(__vcmpeq4(q.y, 0u)) + __popc(__vcmpeq4(q.z, 0u)) +
+                        __popc(__vcmpeq4(q.w, 0u))) >> 3;
+            }
+        } else {
+            for (int64_t t = tid; t < base; t += CB_THREADS) cnt += mask[t] == 0;
+        }
+        before = block_sum(cnt, warp_tot);
+    }
+    // ---- this thread's 16 tokens
+    const int64_t t0 = base + (int64_t)tid * CB_PER_THREAD;
+    unsigned keep = 0;
+#pragma unroll
+    for (int j = 0; j < CB_PER_THREAD; ++j)
+        if (t0 + j < N && (dense || mask[t0 + j] == 0)) keep |= 1u << j;
+    const int mine = __popc(keep);
+    // exclusive scan over the CTA: within the warp, then over the warp totals
+    int incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    int off = before + incl - mine, total = before;
+#pragma unroll
+    for (int w = 0; w < CB_THREADS / 32; ++w) {
+        if (w < warp) off += warp_tot[w];
+        total += warp_tot[w];
+    }
+    int r = off;
+#pragma unroll
+    for (int j = 0; j < CB_PER_THREAD; ++j) {
+        if (t0 + j < N) {
+            if ((keep >> j) & 1u) { idx[r] = (int32_t)(t0 + j); pos[t0 + j] = r; ++r; }
+            else pos[t0 + j] = -1;
+        }
+    }
+    if (blockIdx.x == gridDim.x - 1) {   // the last block knows the total
+        if (tid == 0) status[ST_NK] = total;
+        int64_t end = ((int64_t)total + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
+        if (end > cap) end = cap;
+        for (int64_t q = total + tid; q < end; q += CB_THREADS) idx[q] = 0;
+    }
+}
+
+// One CTA of 1024 threads walks the mask in slabs of 16 x 1024 tokens (inputs too long for the
+// redundant counting above).  Within a slab, token (j, warp, lane) = base + j*1024 + warp*32 + lane;
+// a warp ballot gives each kept token its rank inside its 32-token segment, and an exclusive scan
+// over the 512 segment counts (segments are in ascending token order) gives the segment's offset.
 constexpr int CP_THREADS = 1024;
 constexpr int CP_J = 16;
 
 __global__ void __launch_bounds__(CP_THREADS)
-k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
-          int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
+k_compact_serial(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
+                 int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
 {
     __shared__ int seg[CP_J * 32];
     __shared__ int slab_total;
@@ -67,19 +160,19 @@ k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__res
         carry += slab_total;
         __syncthreads();
     }
-    // padding entries: repeat the first kept token (any valid row)
-    __shared__ int first;
-    if (tid == 0) { first = carry > 0 ? idx[0] : 0; status[ST_NK] = carry; }
-    __syncthreads();
+    if (tid == 0) status[ST_NK] = carry;
     int64_t end = ((int64_t)carry + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
     if (end > cap) end = cap;
-    for (int64_t r = carry + tid; r < end; r += CP_THREADS) idx[r] = first;
+    for (int64_t r = carry + tid; r < end; r += CP_THREADS) idx[r] = 0;
 }
 
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
                            int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s)
 {
-    return launch_pdl(k_compact, dim3(1), dim3(CP_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
+    if (N > CB_MAX_N)
+        return launch_pdl(k_compact_serial, dim3(1), dim3(CP_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
+    const unsigned blocks = (unsigned)((N + CB_TOKENS - 1) / CB_TOKENS);
+    return launch_pdl(k_compact, dim3(blocks), dim3(CB_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
 }
 
 // Row routing.  Unit u < N is token u: a kept token's row goes to dst_compact[pos[u]], a skipped

@@ -236,7 +236,7 @@ static cudaError_t merge_t(const T *X, int64_t n, int C, int k, int dtype, int32
         g.M = (int32_t)n_rest; g.N = k; g.K = C;
         g.status = m.status_k; g.idx = m.kept;
         g.out0 = m.sims; g.ldo = k; g.out_fp32 = 1;
-        g.sk_slots = slots; g.sk_flags = m.status_k + ST_WORDS; g.sk_epoch = 1;
+        g.sk_slots = slots; g.sk_flags = m.status_k + ST_WORDS; g.sk_epoch = 1; g.tune_streamk = -1;
         e = dtype == SKIPFFN_BF16 ? launch_umma_gemm(EPI_PLAIN, g, s) : launch_simt_gemm(EPI_DW, dtype, g, s);
         if (e != cudaSuccess) return e;
     }

@@ -41,6 +41,7 @@
 // reproducible from run to run.
 #include <cuda.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "sched.cuh"
@@ -55,15 +56,28 @@ constexpr int ACC_COLS = 256;                    // fp32 columns per accumulator
 constexpr int TMEM_COLS = 512;
 constexpr int EPI_WARPS = 8;
 constexpr int EPI_BUF_BYTES = 2048;              // per-warp staging: 32 rows x 64 B
+constexpr int X_BUF_BYTES = 4096;                // gate/up: fp32 exchange buffer of a warp pair (32 x 32 words)
 constexpr int UMMA_THREADS = 64 + 32 * EPI_WARPS;
 template <bool PAIR> struct Shape {
     static constexpr int STAGES = PAIR ? 6 : 4;
     static constexpr int B_BYTES = PAIR ? 128 * BK * 2 : 256 * BK * 2;   // B rows staged per CTA
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES +
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_BUF_BYTES + 4 * X_BUF_BYTES +
                                       1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s
+
+// Optional per-role cycle counters (build with -DSKIPFFN_ROLE_CYCLES; never in the default build):
+// every launch adds, per epilogue kind, the cycles its MMA issuers spent waiting for operand
+// stages and for a free accumulator, the producers' waits for free stages, and one epilogue
+// warp's wait and busy time, into status words ST_ROLE_BASE + 8 * EPI + {0..7}.
+#ifdef SKIPFFN_ROLE_CYCLES
+#define ROLE_CLOCK() clock64()
+#define ROLE_ADD(var, t0) (var) += clock64() - (t0)
+#else
+#define ROLE_CLOCK() 0ll
+#define ROLE_ADD(var, t0) (void)(t0)
+#endif
 
 // ------------------------------------------------------------------------------------ PTX
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -169,6 +183,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(c0), "r"(c1), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -225,6 +248,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 lanes x 32 consecutive fp32 columns in the layout of an MMA accumulator fragment: for each
+// group g of 8 columns, thread t receives row t/4, columns 8g + 2(t%4) and +1 in r[4g], r[4g+1] and
+// row t/4 + 8, same columns, in r[4g+2], r[4g+3]
+__device__ __forceinline__ void tmem_ld_frag16(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+// four 8x8 matrices of 16-bit elements between fragment registers and shared memory, transposed:
+// thread t holds elements (row t/4, columns 2(t%4), +1) of each matrix; shared-memory row R (16
+// bytes at the address given by thread 8k + R for matrix k) holds COLUMN R of the matrix
+__device__ __forceinline__ void stsm_x4_trans(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a),
+                 "r"(b), "r"(c), "r"(d)
+                 : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t &a, uint32_t &b, uint32_t &c, uint32_t &d)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(a), "=r"(b), "=r"(c), "=r"(d)
+                 : "r"(addr)
+                 : "memory");
+}
 
 // ---- cluster (SM pair) variants
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -257,6 +310,15 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
         "l"(map), "r"(c0), "r"(c1), "r"(leader_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2,
+                                                 uint32_t leader_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(leader_bar)
         : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols)
@@ -320,7 +382,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int a_mn_major, int b_mn_major
 // ------------------------------------------------------------------------------------ kernel
 struct UmmaParams {
     int32_t M, N, K;                 // host upper bounds
-    int32_t m_from_nk, k_from_nk;    // extent is the device-resident kept count
+    int32_t n_from_nk, k_from_nk;    // extent is the device-resident kept count
     int32_t segments;                // 2: second K segment reads tmA2 / tmB2 (dX)
     int32_t force_bn;                // > 0: tile width override (tuning)
     int32_t force_stages;            // > 0: use fewer ring stages (tuning)
@@ -333,7 +395,7 @@ struct UmmaParams {
     float4 *sk_slots;                // per-CTA partial-accumulator slots
     int32_t *sk_flags;               // SK_FLAGS_PER_CTA flags per slot
     int32_t sk_epoch;                // flag value of this launch
-    int32_t sk_wait_skew;            // 0; test hook: finishing units wait for a value nobody writes
+    int32_t sk_wait_skew;            // 0; debug handles: finishing units wait for a value nobody writes
     // grouped launch (weight gradients): up to three independent problems sharing K; problem g has
     // extents gM[g] x gN[g], operands (tmA, tmB) / (tmA2, tmB2) / (tmA3, tmB2), output gout[g]
     int32_t groups;
@@ -342,10 +404,23 @@ struct UmmaParams {
     int64_t gldo[3];
     int32_t streamk;                 // 0: whole tiles only; else the least number of K-blocks per worker
                                      // that cutting the last waves along K must save to be used
+    // one-instruction operand loads (see TmapSet): which of them the host could encode
+    int32_t a_one, b_one;            // MN-major operand: both 64-wide slabs of a CTA's 128 in one 3-D box
+    int32_t gu_one;                  // gate/up: gate and up rows in one 3-D box; 2 = the up rows come first
+};
+
+// Tensor maps of one launch.  A, B, A2, B2, A3: 2-D maps (box = 64 elements of the contiguous
+// axis x 64 or 128 rows).  Bw, B2w: the same K-major B arrays with 128-row boxes, so that a CTA's
+// whole half of a full-width token tile arrives with one instruction.  A1, A21, A31, B1, B21: 3-D views
+// of MN-major arrays [K rows, 64-wide slab, 64 columns] whose box holds two slabs (128 columns); for
+// gate/up A1 is the 3-D view [K, weight row, {gate, up}] of the two weight matrices.
+struct alignas(64) TmapSet {
+    CUtensorMap A, B, A2, B2, A3, Bw, B2w, A1, A21, A31, B1, B21;
 };
 
 struct alignas(8) SmemCtl {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t xfull[4], xempty[4];    // gate/up epilogue: up-warp -> gate-warp exchange, per warp pair
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -361,6 +436,11 @@ __device__ __forceinline__ void unpack_bf16(uint32_t w, float &lo, float &hi)
     lo = __low2float(v);
     hi = __high2float(v);
 }
+__device__ __forceinline__ unsigned short bf16_bits(float v)
+{
+    return __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ float bf16_from_bits(unsigned short b) { return __uint_as_float((uint32_t)b << 16); }
 
 // sigmoid from the hardware exp2 / reciprocal approximations (relative error ~1e-6, far below the
 // bf16 rounding of everything it feeds)
@@ -373,13 +453,14 @@ __device__ __forceinline__ void fast_swiglu_bwd(float dh, float g, float u, floa
     dg = dh * u * (s * (1.0f + g * (1.0f - s)));
 }
 
-// Epilogue staging.  A warp owns 32 accumulator rows (one per lane).  For a 32-column bf16 chunk
-// each lane holds its row as 16 packed words (64 B).  The rows are written to a 2 KiB per-warp
-// shared-memory buffer (16-byte slots XOR-swizzled by row pair: conflict-free both ways), then read
-// back so that four consecutive lanes cover one row's 64 contiguous bytes: every global store
-// instruction writes eight full 64-byte row segments instead of 32 scattered 16-byte pieces.
-// `my_row` is this lane's destination (row pointer at the chunk's first column) or null for a row
-// that must not be written; `valid_slots` = number of 16-byte slots inside the column range.
+// Epilogue staging of the weight-gradient tiles.  A warp owns 32 accumulator rows (one per lane).
+// For a 32-column bf16 chunk each lane holds its row as 16 packed words (64 B).  The rows are
+// written to a 2 KiB per-warp shared-memory buffer (16-byte slots XOR-swizzled by row pair:
+// conflict-free both ways), then read back so that four consecutive lanes cover one row's 64
+// contiguous bytes: every global store instruction writes eight full 64-byte row segments instead
+// of 32 scattered 16-byte pieces.  `my_row` is this lane's destination (row pointer at the chunk's
+// first column) or null for a row that must not be written; `valid_slots` = number of 16-byte
+// slots inside the column range.
 __device__ __forceinline__ void store_rows_64B(uint32_t sbuf, int lane, const uint32_t (&w)[16],
                                                char *my_row, int valid_slots)
 {
@@ -402,31 +483,6 @@ __device__ __forceinline__ void store_rows_64B(uint32_t sbuf, int lane, const ui
         char *dst = (char *)__shfl_sync(0xffffffffu, (unsigned long long)my_row, row);
         if (dst != nullptr && c < valid_slots) *reinterpret_cast<uint4 *>(dst + c * 16) = v;
     }
-    __syncwarp();
-}
-// The reverse for epilogue inputs.  `v[it]` holds the 16 bytes this lane loaded from row
-// it * 8 + lane / 4, slot lane % 4 (four consecutive lanes cover one row's 64 bytes, so a warp
-// load touches eight full 64-byte segments instead of 32 scattered 16-byte pieces); the same
-// staging buffer turns them into this lane's own row as 16 packed words.
-__device__ __forceinline__ void rows_from_coalesced(uint32_t sbuf, int lane, const uint4 (&v)[4],
-                                                    uint32_t (&w)[16])
-{
-    const int c = lane & 3;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        const int row = it * 8 + (lane >> 2);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sbuf + row * 64 + ((c ^ ((row >> 1) & 3)) << 4)),
-                     "r"(v[it].x), "r"(v[it].y), "r"(v[it].z), "r"(v[it].w)
-                     : "memory");
-    }
-    __syncwarp();
-    const int sw = (lane >> 1) & 3;
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(w[4 * q]), "=r"(w[4 * q + 1]), "=r"(w[4 * q + 2]), "=r"(w[4 * q + 3])
-                     : "r"(sbuf + lane * 64 + ((q ^ sw) << 4))
-                     : "memory");
     __syncwarp();
 }
 // fp32 variant with read-modify-write (dW accumulation): same staging, 16 columns per call
@@ -459,23 +515,110 @@ __device__ __forceinline__ void store_rows_64B_f32(uint32_t sbuf, int lane, cons
     __syncwarp();
 }
 
+// ---- Epilogue staging of the token problems.
+// A warp owns 32 accumulator rows (weight rows) and works on chunks of 32 columns (tokens).  Its
+// accumulator chunk sits in registers as two 16-row MMA fragments: r[16 hb + 4 g + 2 s + e] is row
+// 16 hb + 8 s + t/4, column 8 g + 2 (t%4) + e.  The outputs are token-major ([token, weight row]),
+// i.e. the transpose: one token's 32 weight rows are 64 contiguous bytes.  The transposition runs
+// through a 2 KiB per-warp staging buffer laid out like the output ([32 tokens][64 bytes], 16-byte
+// pieces XOR-swizzled by token pair): stmatrix / ldmatrix with .trans move whole 8x8 blocks
+// between fragments and the buffer, and global memory is touched with 16-byte accesses, four
+// consecutive lanes covering one token's 64 bytes.
+__device__ __forceinline__ uint32_t stage_addr(uint32_t sbuf, int token, int piece)
+{
+    return sbuf + token * 64 + ((piece ^ ((token >> 1) & 3)) << 4);
+}
+// packed fragment P[8 hb + 2 g + s] = (column 8g + 2(t%4) low half, +1 high half) of row block (hb, s)
+__device__ __forceinline__ void frag_to_stage(uint32_t sbuf, int lane, const uint32_t (&P)[16])
+{
+    const int k = lane >> 3, rr = lane & 7;
+#pragma unroll
+    for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+        for (int g0 = 0; g0 < 4; g0 += 2) {
+            const int token = 8 * (g0 + (k >> 1)) + rr, piece = 2 * hb + (k & 1);
+            stsm_x4_trans(stage_addr(sbuf, token, piece), P[8 * hb + 2 * g0], P[8 * hb + 2 * g0 + 1],
+                          P[8 * hb + 2 * g0 + 2], P[8 * hb + 2 * g0 + 3]);
+        }
+}
+__device__ __forceinline__ void stage_to_frag(uint32_t sbuf, int lane, uint32_t (&P)[16])
+{
+    const int k = lane >> 3, rr = lane & 7;
+#pragma unroll
+    for (int hb = 0; hb < 2; ++hb)
+#pragma unroll
+        for (int g0 = 0; g0 < 4; g0 += 2) {
+            const int token = 8 * (g0 + (k >> 1)) + rr, piece = 2 * hb + (k & 1);
+            ldsm_x4_trans(stage_addr(sbuf, token, piece), P[8 * hb + 2 * g0], P[8 * hb + 2 * g0 + 1],
+                          P[8 * hb + 2 * g0 + 2], P[8 * hb + 2 * g0 + 3]);
+        }
+}
+// Staging buffer -> global: lane L moves, for it = 0..3, the 16-byte piece L%4 of token 8 it + L/4 to
+// dst[it] (this lane's address inside that token's row, or null).
+__device__ __forceinline__ void stage_to_global(uint32_t sbuf, int lane, char *const (&dst)[4])
+{
+    __syncwarp();
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int token = it * 8 + (lane >> 2);
+        uint4 v;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                     : "r"(stage_addr(sbuf, token, lane & 3))
+                     : "memory");
+        if (dst[it] != nullptr) *reinterpret_cast<uint4 *>(dst[it]) = v;
+    }
+    __syncwarp();
+}
+// Global -> staging buffer (zeros where src[it] is null), then into fragment registers.
+__device__ __forceinline__ void global_to_frag(uint32_t sbuf, int lane, const char *const (&src)[4], uint32_t (&P)[16])
+{
+    uint4 v[4];
+#pragma unroll
+    for (int it = 0; it < 4; ++it)
+        v[it] = src[it] != nullptr ? __ldcs(reinterpret_cast<const uint4 *>(src[it])) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int token = it * 8 + (lane >> 2);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_addr(sbuf, token, lane & 3)), "r"(v[it].x),
+                     "r"(v[it].y), "r"(v[it].z), "r"(v[it].w)
+                     : "memory");
+    }
+    __syncwarp();
+    stage_to_frag(sbuf, lane, P);
+    __syncwarp();
+}
+
+// Two kinds of problems share the kernel.
+//   Token problems (gate/up, down, dH, dX): the WEIGHT rows run along the accumulator rows (MMA M,
+//   256 per SM pair) and the kept TOKENS along the accumulator columns (MMA N, any multiple of 16
+//   up to 256), so a kept count that is not a multiple of the tile width costs at most 15 padded
+//   columns instead of up to 255 padded rows.  A = weights (K-major or MN-major), B = compacted
+//   token rows (K-major).  The outputs are token-major arrays [token, weight row]: for one token
+//   the 32 lanes of a warp hold 32 consecutive weight rows, i.e. 64 contiguous bytes of its
+//   output row, so every epilogue load / store instruction moves one full 64-byte segment.
+//   Weight-gradient problems (and the plain GEMM of the token merge): both axes are weight axes,
+//   K is the kept count; tiles are 256 x 256 and rows are staged through shared memory.
 template <int EPI, bool A_MN, bool B_MN, bool PAIR>
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
-k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
-            const __grid_constant__ CUtensorMap tmA3, const UmmaParams p)
+k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
 {
+    const CUtensorMap &tmA = tm.A, &tmB = tm.B, &tmA2 = tm.A2, &tmB2 = tm.B2, &tmA3 = tm.A3;
     constexpr bool GATEUP = (EPI == EPI_GATEUP);
+    constexpr bool TOK = (EPI != EPI_DW);         // token problem: tokens on the accumulator columns
     constexpr int STAGES = Shape<PAIR>::STAGES;
     constexpr int STAGE_BYTES = Shape<PAIR>::STAGE_BYTES;
     constexpr int SPLIT = PAIR ? 2 : 1;           // CTAs sharing one tile
-    constexpr int TILE_M = BM * SPLIT;
+    constexpr int TILE_M = BM * SPLIT;            // accumulator rows of one tile
+    // gate/up: each CTA's 128 rows are 64 gate rows followed by the 64 up rows of the same
+    // intermediate indices, so a tile covers TILE_M / 2 indices
+    constexpr int M_UNIT = GATEUP ? TILE_M / 2 : TILE_M;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t epi_bufs = tiles + STAGES * STAGE_BYTES;
     SmemCtl *ctl = reinterpret_cast<SmemCtl *>(smem_raw + (tiles - raw) + STAGES * STAGE_BYTES +
-                                               EPI_WARPS * EPI_BUF_BYTES);
+                                               EPI_WARPS * EPI_BUF_BYTES + 4 * X_BUF_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // position in the SM pair; 0 leads
@@ -490,6 +633,10 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&ctl->tmem_full[s]), 1);
             mbar_init(smem_u32(&ctl->tmem_empty[s]), EPI_WARPS * SPLIT);
+        }
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(smem_u32(&ctl->xfull[s]), 1);
+            mbar_init(smem_u32(&ctl->xempty[s]), 1);
         }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -510,32 +657,42 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int nk = p.status[ST_NK];
-    const int M = p.m_from_nk ? nk : p.M;
     const int K = p.k_from_nk ? nk : p.K;
-    // accumulator columns per tile (256 unless overridden); gate and up halves share a tile, so its
-    // output is half as wide
-    const int bn = (GATEUP || p.force_bn <= 0) ? BN : p.force_bn;
-    const int n_tile = GATEUP ? BN / 2 : bn;
-    // tiles of problem g: ids [g_first[g], g_first[g+1]), the row-tile index running fastest
-    const int groups = (EPI == EPI_DW) ? p.groups : 1;
+    // token problems: the column extent is the kept count rounded up to the MMA's N granularity;
+    // columns nk .. n_tot-1 exist only as padding (their operand rows are zero)
+    const int n_tot = TOK ? (p.n_from_nk ? ((nk + 15) & ~15) : p.N) : 0;
+    // accumulator columns per tile (256 unless overridden)
+    const int tile_w = p.force_bn > 0 ? p.force_bn : BN;
+    // tiles of problem g: ids [g_first[g], g_first[g+1]); token problems run the column (token)
+    // tile index fastest, so that tiles sharing a weight panel run at the same time
+    const int groups = TOK ? 1 : p.groups;
     int g_m[3], g_n[3], g_num_m[3], g_first[4];
     g_first[0] = 0;
 #pragma unroll
     for (int g = 0; g < 3; ++g) {
-        g_m[g] = g < groups ? ((EPI == EPI_DW) ? p.gM[g] : M) : 0;
-        g_n[g] = g < groups ? ((EPI == EPI_DW) ? p.gN[g] : p.N) : 0;
-        g_num_m[g] = (g_m[g] + TILE_M - 1) / TILE_M;
-        g_first[g + 1] = g_first[g] + g_num_m[g] * ((g_n[g] + n_tile - 1) / n_tile);
+        g_m[g] = g < groups ? (TOK ? p.M : p.gM[g]) : 0;
+        g_n[g] = g < groups ? (TOK ? n_tot : p.gN[g]) : 0;
+        g_num_m[g] = (g_m[g] + M_UNIT - 1) / M_UNIT;
+        g_first[g + 1] = g_first[g] + g_num_m[g] * ((g_n[g] + tile_w - 1) / tile_w);
     }
     const int num_tiles = g_first[3];
+    const int num_n0 = (g_n[0] + tile_w - 1) / tile_w;
     auto pick = [](const int (&a)[3], int g) { return g == 2 ? a[2] : (g == 1 ? a[1] : a[0]); };
-    struct TileLoc { int g, m0, n0; };
+    struct TileLoc { int g, m0, n0, bn; };   // m0 in units of output rows (gate/up: intermediate indices)
     auto locate = [&](int tile) {
         TileLoc t;
-        t.g = (EPI == EPI_DW) ? (tile >= g_first[2] ? 2 : (tile >= g_first[1] ? 1 : 0)) : 0;
-        const int local = tile - (t.g == 2 ? g_first[2] : (t.g == 1 ? g_first[1] : 0)), nm = pick(g_num_m, t.g);
-        t.m0 = (local % nm) * TILE_M;
-        t.n0 = (local / nm) * n_tile;
+        if (TOK) {
+            t.g = 0;
+            t.m0 = (tile / num_n0) * M_UNIT;
+            t.n0 = (tile % num_n0) * tile_w;
+            t.bn = min(tile_w, n_tot - t.n0);
+        } else {
+            t.g = tile >= g_first[2] ? 2 : (tile >= g_first[1] ? 1 : 0);
+            const int local = tile - (t.g == 2 ? g_first[2] : (t.g == 1 ? g_first[1] : 0)), nm = pick(g_num_m, t.g);
+            t.m0 = (local % nm) * TILE_M;
+            t.n0 = (local / nm) * tile_w;
+            t.bn = tile_w;
+        }
         return t;
     };
     const int kb_per_seg = (K + BK - 1) / BK;
@@ -550,102 +707,135 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                          (long long)(num_workers - rem_tiles) * num_kb >= (long long)p.streamk * num_workers;
     sched.init(worker, num_workers, num_tiles, num_kb, split_k);
     const int num_segs = sched.count();
-    const int bn_cta = bn / SPLIT;         // B rows (tile columns) this CTA stages
-    const int b_slabs = (bn_cta + 63) / 64;
     const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
-
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0 && !zero_acc) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmB);
-            if (GATEUP || p.segments == 2 || groups > 1) prefetch_tmap(&tmB2);
-            if (p.segments == 2 || groups > 1) prefetch_tmap(&tmA2);
+            if (p.segments == 2 || groups > 1) prefetch_tmap(&tmB2);
+            if (GATEUP || p.segments == 2 || groups > 1) prefetch_tmap(&tmA2);
             if (groups > 2) prefetch_tmap(&tmA3);
-            // bytes landing on the (leader's) full barrier per stage, from every CTA of the tile
-            const uint32_t stage_tx = SPLIT * (A_BYTES + b_slabs * CHUNK_BYTES);
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            // TMA loads of one K-block of one run into ring stage `stage`
-            auto issue = [&](const Seg &sg, int kb) {
-                const int tile = sg.tile;
-                const TileLoc tl = locate(tile);
-                const int m0 = tl.m0 + (int)rank * BM, n0 = tl.n0;
-                const int nb0 = GATEUP ? n0 : n0 + (int)rank * bn_cta;   // first B row of this CTA
-                const int seg = kb >= kb_per_seg ? 1 : 0;
-                const int k0 = (kb - seg * kb_per_seg) * BK;
-                const CUtensorMap *mA = tl.g == 2 ? &tmA3 : ((tl.g == 1 || seg) ? &tmA2 : &tmA);
-                const CUtensorMap *mB = (tl.g >= 1 || seg) ? &tmB2 : &tmB;
-                const uint32_t own_bar = smem_u32(&ctl->full[stage]);
-                const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
-                const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                auto load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1) {
-                    if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar);
-                    else tma_load_2d(dst, map, c0, c1, bar);
-                };
-                if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
-                if (A_MN) {
-#pragma unroll
-                    for (int j = 0; j < BM / 64; ++j) load(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0);
-                } else {
-                    load(sa, mA, k0, m0);
-                }
-                if (B_MN) {          // 64-column slabs of BK rows
-                    for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, nb0 + 64 * j, k0);
-                } else if (GATEUP && PAIR) {   // leader stages the 128 gate rows, its peer the up rows
-#pragma unroll
-                    for (int j = 0; j < 2; ++j)
-                        load(sb + j * CHUNK_BYTES, rank == 0 ? &tmB : &tmB2, k0, n0 + 64 * j);
-                } else if (GATEUP) { // 128 gate rows, then 128 up rows, in 64-row pieces
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        load(sb + j * CHUNK_BYTES, &tmB, k0, n0 + 64 * j);
-                        load(sb + (2 + j) * CHUNK_BYTES, &tmB2, k0, n0 + 64 * j);
-                    }
-                } else {             // 64-row pieces of a K-major tile are contiguous in smem
-                    for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
-                }
-            };
+            long long role_a = 0;
             for (int si = 0; ok && si < num_segs; ++si) {
                 const Seg sg = sched.get(si);
+                const TileLoc tl = locate(sg.tile);
+                const int bn_cta = tl.bn / SPLIT;          // B rows (tile columns) this CTA stages
+                const int b_slabs = (bn_cta + 63) / 64;
+                // bytes landing on the (leader's) full barrier per stage, from every CTA of the tile
+                const uint32_t stage_tx = SPLIT * (A_BYTES + b_slabs * CHUNK_BYTES);
+                const int m0 = GATEUP ? tl.m0 + (int)rank * (BM / 2) : tl.m0 + (int)rank * BM;
+                const int nb0 = tl.n0 + (int)rank * bn_cta;   // first B row of this CTA
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    const long long tw = ROLE_CLOCK();
                     ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status,
                                    SITE_PRODUCER_EMPTY);
+                    ROLE_ADD(role_a, tw);
                     if (!ok) break;
-                    issue(sg, kb);
+                    const int seg = kb >= kb_per_seg ? 1 : 0;
+                    const int k0 = (kb - seg * kb_per_seg) * BK;
+                    const CUtensorMap *mA = tl.g == 2 ? &tmA3 : ((tl.g == 1 || seg) ? &tmA2 : &tmA);
+                    const CUtensorMap *mB = (tl.g >= 1 || seg) ? &tmB2 : &tmB;
+                    const uint32_t own_bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    auto load = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1) {
+                        if (PAIR) tma_load_2d_pair(dst, map, c0, c1, bar);
+                        else tma_load_2d(dst, map, c0, c1, bar);
+                    };
+                    auto load3 = [&](uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2) {
+                        if (PAIR) tma_load_3d_pair(dst, map, c0, c1, c2, bar);
+                        else tma_load_3d(dst, map, c0, c1, c2, bar);
+                    };
+                    if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
+                    if (GATEUP) {        // 64 gate rows and the 64 up rows of the same indices
+                        if (p.gu_one) {
+                            load3(sa, &tm.A1, k0, m0, 0);
+                        } else {
+                            load(sa, &tmA, k0, m0);
+                            load(sa + CHUNK_BYTES, &tmA2, k0, m0);
+                        }
+                    } else if (A_MN) {
+                        if (p.a_one) {
+                            load3(sa, tl.g == 2 ? &tm.A31 : ((tl.g == 1 || seg) ? &tm.A21 : &tm.A1), 0, k0, m0 >> 6);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < BM / 64; ++j) load(sa + j * CHUNK_BYTES, mA, m0 + 64 * j, k0);
+                        }
+                    } else {
+                        load(sa, mA, k0, m0);
+                    }
+                    if (B_MN) {          // 64-column slabs of BK rows
+                        if (p.b_one && bn_cta == 128) {
+                            load3(sb, (tl.g >= 1 || seg) ? &tm.B21 : &tm.B1, 0, k0, nb0 >> 6);
+                        } else {
+                            for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, nb0 + 64 * j, k0);
+                        }
+                    } else if (TOK) {    // K-major token rows: boxes of 128 rows, then one of 64 if 64 are left
+                        int j = 0;
+                        for (; b_slabs - j > 1; j += 2) load(sb + j * CHUNK_BYTES, seg ? &tm.B2w : &tm.Bw, k0, nb0 + 64 * j);
+                        if (j < b_slabs) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
+                    } else {             // 64-row pieces of a K-major tile are contiguous in smem
+                        for (int j = 0; j < b_slabs; ++j) load(sb + j * CHUNK_BYTES, mB, k0, nb0 + 64 * j);
+                    }
                     if (++stage == nst) { stage = 0; phase ^= 1; }
                 }
             }
+#ifdef SKIPFFN_ROLE_CYCLES
+            if (rank == 0) atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 3], (int)(role_a >> 4));
+#endif
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && !zero_acc && rank == 0) {
-            const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, TILE_M, bn);
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
+            // shared-memory descriptors of ring stage 0; a K step of 16 elements advances the address
+            // field by 32 bytes (K-major) or by 16 rows of 128 bytes (MN-major)
+            constexpr uint32_t KINC_A = A_MN ? (UMMA_K * 128) >> 4 : (UMMA_K * 2) >> 4;
+            constexpr uint32_t KINC_B = B_MN ? (UMMA_K * 128) >> 4 : (UMMA_K * 2) >> 4;
+            const uint64_t da0 = A_MN ? make_desc(tiles, CHUNK_BYTES, 1024) : make_desc(tiles, 16, 1024);
+            const uint64_t db0 = B_MN ? make_desc(tiles + A_BYTES, CHUNK_BYTES, 1024) : make_desc(tiles + A_BYTES, 16, 1024);
+            const int k_tail = K - (kb_per_seg - 1) * BK;   // elements in the last K-block
+            const int k_steps_last = k_tail < BK ? (k_tail + UMMA_K - 1) / UMMA_K : BK / UMMA_K;
+            long long role_full = 0, role_acc = 0;
+            const long long role_t0 = ROLE_CLOCK();
             for (int si = 0; ok && si < num_segs; ++si) {
                 const Seg sg = sched.get(si);
+                const TileLoc tl = locate(sg.tile);
+                const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, TILE_M, tl.bn);
+                const long long ta = ROLE_CLOCK();
                 ok = mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1, abort_flag, p.status,
                                SITE_MMA_TMEM_EMPTY);
+                ROLE_ADD(role_acc, ta);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * ACC_COLS;
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    const long long tf = ROLE_CLOCK();
                     ok = mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag, p.status,
                                    SITE_MMA_FULL);
+                    ROLE_ADD(role_full, tf);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    // descriptors of this stage: the ring base descriptors plus the stage offset in the
+                    // 14-bit address field (shared memory ends below 256 KiB, so no carry leaves the field)
+                    const uint64_t da = da0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                    const uint64_t db = db0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+                    // A reduction over kept tokens ends inside its last K-block: rows past the
+                    // count (rounded up to 16, zero up to there) hold stale data and stay unread
+                    int k_steps = BK / UMMA_K;
+                    if (!TOK && p.k_from_nk && kb == kb_per_seg - 1) k_steps = k_steps_last;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t da = A_MN ? make_desc(sa + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
-                                                 : make_desc(sa + k * (UMMA_K * 2), 16, 1024);
-                        const uint64_t db = B_MN ? make_desc(sb + k * (UMMA_K * 128), CHUNK_BYTES, 1024)
-                                                 : make_desc(sb + k * (UMMA_K * 2), 16, 1024);
-                        const uint32_t accumulate = (kb != sg.kb0 || k != 0);   // first MMA of a run overwrites
-                        if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, accumulate);
-                        else umma_bf16(d_tmem, da, db, idesc, accumulate);
+                        if (k < k_steps) {
+                            const uint32_t accumulate = (kb != sg.kb0 || k != 0);   // first MMA of a run overwrites
+                            if (PAIR) umma_bf16_pair(d_tmem, da + (uint64_t)(k * KINC_A), db + (uint64_t)(k * KINC_B), idesc, accumulate);
+                            else umma_bf16(d_tmem, da + (uint64_t)(k * KINC_A), db + (uint64_t)(k * KINC_B), idesc, accumulate);
+                        }
                     }
                     // the stage is reusable (in both CTAs) once these MMAs retire
                     if (PAIR) umma_commit_pair(smem_u32(&ctl->empty[stage]));
@@ -658,6 +848,12 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1; }
             }
+#ifdef SKIPFFN_ROLE_CYCLES
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 0], (int)(role_full >> 4));
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 1], (int)(role_acc >> 4));
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 2], (int)((clock64() - role_t0) >> 4));
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 7], 1);
+#endif
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -670,6 +866,14 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int esz = p.out_fp32 ? 4 : 2;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
+        long long role_wait = 0;
+        const long long role_e0 = ROLE_CLOCK();
+        // gate/up: warps of quarters 0, 1 hold gate rows, quarters 2, 3 the up rows of the same
+        // indices; pair x = (quarter & 1) + 2 * half exchanges the up values through shared memory
+        const int xpair = (quarter & 1) + 2 * half;
+        const uint32_t xbuf = epi_bufs + EPI_WARPS * EPI_BUF_BYTES + xpair * X_BUF_BYTES;
+        const uint32_t xfull_bar = smem_u32(&ctl->xfull[xpair]), xempty_bar = smem_u32(&ctl->xempty[xpair]);
+        uint32_t xcount = 0;            // chunks exchanged so far by this warp
         // accumulators are handed back on the leader's barrier, which its MMA warp waits on
         const uint32_t empty_bar0 = smem_u32(&ctl->tmem_empty[0]);
         // hand-over slots: a warp reads back exactly the words the same warp of the producing CTA wrote
@@ -679,9 +883,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         };
         for (int si = 0; ok && si < num_segs; ++si) {
             const Seg sg = sched.get(si);
-            const int tile = sg.tile;
-            const TileLoc tl = locate(tile);
-            const int m0 = tl.m0 + (int)rank * BM, n0 = tl.n0;
+            const TileLoc tl = locate(sg.tile);
+            const int n0 = tl.n0, bn = tl.bn;
             if (sg.partial) {
                 // ---- this run ends before the tile does: park the raw accumulator in this CTA's slot
                 ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
@@ -692,7 +895,8 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll 1
                 for (int col = half * 32, j = 0; col < bn; col += 64, ++j) {
                     uint32_t r[32];
-                    tmem_ld32(t_acc + col, r);
+                    if (TOK) { tmem_ld_frag16(t_acc + col, r); tmem_ld_frag16(t_acc + (16u << 16) + col, r + 16); }
+                    else tmem_ld32(t_acc + col, r);
                     tmem_ld_wait();
                     float4 *dst = slot_ptr(my_slot, j);
 #pragma unroll
@@ -715,34 +919,17 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 continue;
             }
             const bool add_slots = sg.kb0 > 0;
-            const int m = m0 + row_in_tile;
-            const int n_end = min(n0 + n_tile, pick(g_n, tl.g));
+            // this lane's output row: a weight row of the problem (token problems) or a row of the
+            // weight gradient
+            const bool is_up = GATEUP && ((quarter >= 2) != (p.gu_one == 2));
+            const int m = GATEUP ? tl.m0 + (int)rank * (BM / 2) + (quarter & 1) * 32 + lane
+                                 : tl.m0 + (int)rank * BM + row_in_tile;
             const bool row_valid = m < pick(g_m, tl.g);
-            int64_t tok = 0;
-            if ((EPI == EPI_DOWN || EPI == EPI_DX) && row_valid) tok = p.idx[m];
-            // prefetch of the per-row epilogue inputs of the first chunk (overlaps the accumulator wait)
-            uint4 pa[4], pb[4];
-            auto prefetch = [&](int n) {
-                // compact rows m0 + quarter * 32 .. + 31 of in0 / in1, loaded eight rows per instruction
-                if ((EPI == EPI_DH || EPI == EPI_DOWN || EPI == EPI_DX) && p.in0 != nullptr) {
-                    const int c = lane & 3;
-#pragma unroll
-                    for (int it = 0; it < 4; ++it) {
-                        const int mr = m0 + quarter * 32 + it * 8 + (lane >> 2);
-                        pa[it] = make_uint4(0, 0, 0, 0);
-                        pb[it] = make_uint4(0, 0, 0, 0);
-                        if (mr < pick(g_m, tl.g) && n + c * 8 < n_end) {
-                            const int64_t o = (int64_t)mr * p.ldo + n + c * 8;
-                            pa[it] = __ldcs(reinterpret_cast<const uint4 *>((const bf16 *)p.in0 + o));
-                            if (EPI == EPI_DH) pb[it] = __ldcs(reinterpret_cast<const uint4 *>((const bf16 *)p.in1 + o));
-                        }
-                    }
-                }
-            };
-            prefetch(n0 + half * 32);
             if (!zero_acc) {
+                const long long tw = ROLE_CLOCK();
                 ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
                                SITE_EPI_TMEM_FULL);
+                ROLE_ADD(role_wait, tw);
                 if (!ok) break;
                 tc_fence_after();
             }
@@ -756,23 +943,20 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 if (!ok) break;
             }
+            const int n_end = TOK ? n0 + bn : min(n0 + bn, pick(g_n, tl.g));
 
 #pragma unroll 1
             for (int n = n0 + half * 32; n < n_end; n += 64) {
                 const int col = n - n0;
-                uint32_t r[32], r2[GATEUP ? 32 : 1];
+                uint32_t r[32];
                 if (!zero_acc) {
-                    tmem_ld32(t_row + col, r);
-                    if (GATEUP) tmem_ld32(t_row + BN / 2 + col, *reinterpret_cast<uint32_t(*)[32]>(&r2));
+                    if (TOK) { tmem_ld_frag16(t_row + col, r); tmem_ld_frag16(t_row + (16u << 16) + col, r + 16); }
+                    else tmem_ld32(t_row + col, r);
+                    tmem_ld_wait();
                 } else {
 #pragma unroll
                     for (int q = 0; q < 32; ++q) r[q] = 0u;
                 }
-                uint4 ca[4], cb[4];
-#pragma unroll
-                for (int v = 0; v < 4; ++v) { ca[v] = pa[v]; cb[v] = pb[v]; }
-                if (n + 64 < n_end) prefetch(n + 64);
-                if (!zero_acc) tmem_ld_wait();
                 if (add_slots) {
                     const int j = col >> 6;   // this warp's j-th 32-column chunk of the accumulator
                     for (int q = sg.src_lo; q < worker; ++q) {
@@ -786,85 +970,154 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + a.z);
                             r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + a.w);
                         }
-                        if (GATEUP) {   // the up half of the accumulator: columns 128 + col
-                            const float4 *src2 = slot_ptr(q * SPLIT + (int)rank, j + 2);
-#pragma unroll
-                            for (int v = 0; v < 8; ++v) {
-                                const float4 a = __ldcg(src2 + v * 32);
-                                r2[GATEUP ? 4 * v : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v : 0]) + a.x);
-                                r2[GATEUP ? 4 * v + 1 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 1 : 0]) + a.y);
-                                r2[GATEUP ? 4 * v + 2 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 2 : 0]) + a.z);
-                                r2[GATEUP ? 4 * v + 3 : 0] = __float_as_uint(__uint_as_float(r2[GATEUP ? 4 * v + 3 : 0]) + a.w);
-                            }
-                        }
                     }
                 }
-                const int valid_slots = min(4, (n_end - n) / 8);
-                uint32_t w[16];
-                if (EPI == EPI_GATEUP) {
-                    // compacted G, U, H; rows past Nk inside the tile are written as zeros
-                    const int64_t o = (int64_t)m * p.ldo + n;
-                    char *rowG = (char *)((bf16 *)p.out0 + o), *rowU = (char *)((bf16 *)p.out1 + o),
-                         *rowH = (char *)((bf16 *)p.out2 + o);
-                    if (!row_valid) {
+                if (TOK) {
+                    // ---- token problems: column c of the chunk is token n + c.  Tokens below nk are
+                    // real; tokens nk .. n_end-1 are the padding of the last tile (stored as zeros
+                    // where a later reduction over tokens reads them).  r[] is in fragment layout:
+                    // r[16 hb + 4 g + 2 s + e] = row 16 hb + 8 s + lane/4, column 8 g + 2 (lane%4) + e.
+                    const int cols = min(32, n_end - n);          // columns of this chunk inside the tile
+                    const int real = max(0, min(cols, nk - n));   // of which real tokens
+                    const int fc = (lane & 3) * 2;                // this thread's first column in a group of 8
+                    // 16-byte pieces: lane moves piece lane%4 (8 weight rows) of tokens 8 it + lane/4
+                    const int m_warp = m - lane;                  // first weight row of this warp
+                    const bool piece_ok = m_warp + 8 * (lane & 3) < pick(g_m, tl.g);
+                    const int64_t piece_off = (int64_t)m_warp + 8 * (lane & 3);
+                    auto tok_of = [&](int it) { return it * 8 + (lane >> 2); };
+                    // zero the accumulator columns that are padding (so every derived value is zero)
+                    if (real < cols) {
 #pragma unroll
-                        for (int q = 0; q < 32; ++q) { r[q] = 0u; r2[GATEUP ? q : 0] = 0u; }
+                        for (int q = 0; q < 32; ++q)
+                            if (8 * ((q >> 2) & 3) + fc + (q & 1) >= real) r[q] = 0u;
                     }
+                    if (EPI == EPI_GATEUP) {
+                        char *dst[4];
+                        const uint32_t xslot = xbuf + lane * 16;
+                        if (is_up) {
+                            // hand the fp32 up values to the gate warp (same fragment layout there), then store U
+                            ok = mbar_wait(xempty_bar, (xcount & 1) ^ 1, abort_flag, p.status, SITE_EPI_EXCHANGE);
+                            if (!ok) break;
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) w[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
-                    store_rows_64B(sbuf, lane, w, rowG, valid_slots);
+                            for (int v = 0; v < 8; ++v)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xslot + v * 512), "r"(r[4 * v]),
+                                             "r"(r[4 * v + 1]), "r"(r[4 * v + 2]), "r"(r[4 * v + 3])
+                                             : "memory");
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(xfull_bar);
+                            if (p.out1 != nullptr) {
+                                uint32_t P[16];
 #pragma unroll
-                    for (int q = 0; q < 16; ++q)
-                        w[q] = pack_bf16(__uint_as_float(r2[GATEUP ? 2 * q : 0]), __uint_as_float(r2[GATEUP ? 2 * q + 1 : 0]));
-                    store_rows_64B(sbuf, lane, w, rowU, valid_slots);
+                                for (int q = 0; q < 16; ++q) P[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+                                frag_to_stage(sbuf, lane, P);
 #pragma unroll
-                    for (int q = 0; q < 16; ++q)
-                        w[q] = pack_bf16(fast_swiglu(__uint_as_float(r[2 * q]), __uint_as_float(r2[GATEUP ? 2 * q : 0])),
-                                         fast_swiglu(__uint_as_float(r[2 * q + 1]), __uint_as_float(r2[GATEUP ? 2 * q + 1 : 0])));
-                    store_rows_64B(sbuf, lane, w, rowH, valid_slots);
-                } else if (EPI == EPI_DX && p.out_fp32) {
-                    // pre-norm variant: the raw fp32 gradient w.r.t. the normalised rows, compact,
-                    // no residual (the normalisation's backward runs afterwards, row-wide)
-                    char *row = row_valid ? (char *)p.out0 + ((int64_t)m * p.ldo + n) * 4 : nullptr;
+                                for (int it = 0; it < 4; ++it)
+                                    dst[it] = (tok_of(it) < cols && piece_ok)
+                                                  ? (char *)((bf16 *)p.out1 + (int64_t)(n + tok_of(it)) * p.ldo + piece_off) : nullptr;
+                                stage_to_global(sbuf, lane, dst);
+                            }
+                        } else {
+                            ok = mbar_wait(xfull_bar, xcount & 1, abort_flag, p.status, SITE_EPI_EXCHANGE);
+                            if (!ok) break;
+                            uint32_t u[32];
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
+                            for (int v = 0; v < 8; ++v)
+                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(u[4 * v]), "=r"(u[4 * v + 1]), "=r"(u[4 * v + 2]), "=r"(u[4 * v + 3])
+                                             : "r"(xslot + v * 512)
+                                             : "memory");
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(xempty_bar);
+                            uint32_t P[16];
+                            if (p.out0 != nullptr) {
 #pragma unroll
-                        for (int q = 0; q < 16; ++q) w[q] = r[hh * 16 + q];
-                        store_rows_64B_f32(sbuf, lane, w, row ? row + hh * 64 : nullptr,
-                                           min(4, max(0, (n_end - n - hh * 16) / 4)), 0);
+                                for (int q = 0; q < 16; ++q) P[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+                                frag_to_stage(sbuf, lane, P);
+#pragma unroll
+                                for (int it = 0; it < 4; ++it)
+                                    dst[it] = (tok_of(it) < cols && piece_ok)
+                                                  ? (char *)((bf16 *)p.out0 + (int64_t)(n + tok_of(it)) * p.ldo + piece_off) : nullptr;
+                                stage_to_global(sbuf, lane, dst);
+                            }
+#pragma unroll
+                            for (int q = 0; q < 16; ++q)
+                                P[q] = pack_bf16(fast_swiglu(__uint_as_float(r[2 * q]), __uint_as_float(u[2 * q])),
+                                                 fast_swiglu(__uint_as_float(r[2 * q + 1]), __uint_as_float(u[2 * q + 1])));
+                            frag_to_stage(sbuf, lane, P);
+#pragma unroll
+                            for (int it = 0; it < 4; ++it)
+                                dst[it] = (tok_of(it) < cols && piece_ok)
+                                              ? (char *)((bf16 *)p.out2 + (int64_t)(n + tok_of(it)) * p.ldo + piece_off) : nullptr;
+                            stage_to_global(sbuf, lane, dst);
+                        }
+                        ++xcount;
+                    } else if (EPI == EPI_DX && p.out_fp32) {
+                        // pre-norm variant: the raw fp32 gradient w.r.t. the normalised rows, compact,
+                        // no residual (the normalisation's backward runs afterwards, row-wide); two
+                        // consecutive tokens per thread, 4-byte stores
+                        float *Y = (float *)p.out0 + (int64_t)n * p.ldo + m_warp;
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) {
+                            const int row = 16 * (q >> 4) + 8 * ((q >> 1) & 1) + (lane >> 2);
+                            const int c = 8 * ((q >> 2) & 3) + fc + (q & 1);
+                            if (c < real && m_warp + row < pick(g_m, tl.g)) Y[(int64_t)c * p.ldo + row] = __uint_as_float(r[q]);
+                        }
+                    } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
+                        // residual add in fp32, one rounding, scatter to the token's row
+                        const char *src[4];
+                        char *dst[4];
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) {
+                            const bool v = tok_of(it) < real && piece_ok;
+                            src[it] = v ? (const char *)((const bf16 *)p.in0 + (int64_t)(n + tok_of(it)) * p.ldo + piece_off) : nullptr;
+                            dst[it] = v ? (char *)((bf16 *)p.out0 + (int64_t)p.idx[n + tok_of(it)] * p.ldo + piece_off) : nullptr;
+                        }
+                        uint32_t R[16], P[16];
+                        global_to_frag(sbuf, lane, src, R);
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            float a0, a1;
+                            unpack_bf16(R[q], a0, a1);
+                            P[q] = pack_bf16(a0 + __uint_as_float(r[2 * q]), a1 + __uint_as_float(r[2 * q + 1]));
+                        }
+                        frag_to_stage(sbuf, lane, P);
+                        stage_to_global(sbuf, lane, dst);
+                    } else if (EPI == EPI_DH) {
+                        const char *src[4];
+                        char *dst[4];
+                        int64_t off[4];
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) off[it] = ((int64_t)(n + tok_of(it)) * p.ldo + piece_off) * 2;
+                        uint32_t Gf[16], Uf[16], P[16], Q[16];
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) src[it] = (tok_of(it) < real && piece_ok) ? (const char *)p.in0 + off[it] : nullptr;
+                        global_to_frag(sbuf, lane, src, Gf);
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) src[it] = (tok_of(it) < real && piece_ok) ? (const char *)p.in1 + off[it] : nullptr;
+                        global_to_frag(sbuf, lane, src, Uf);
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            float g0, g1, u0, u1, dg0, dg1, du0, du1;
+                            unpack_bf16(Gf[q], g0, g1);
+                            unpack_bf16(Uf[q], u0, u1);
+                            fast_swiglu_bwd(__uint_as_float(r[2 * q]), g0, u0, dg0, du0);
+                            fast_swiglu_bwd(__uint_as_float(r[2 * q + 1]), g1, u1, dg1, du1);
+                            P[q] = pack_bf16(dg0, dg1);
+                            Q[q] = pack_bf16(du0, du1);
+                        }
+                        frag_to_stage(sbuf, lane, P);
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) dst[it] = (tok_of(it) < cols && piece_ok) ? (char *)p.out0 + off[it] : nullptr;
+                        stage_to_global(sbuf, lane, dst);
+                        frag_to_stage(sbuf, lane, Q);
+#pragma unroll
+                        for (int it = 0; it < 4; ++it) dst[it] = (tok_of(it) < cols && piece_ok) ? (char *)p.out1 + off[it] : nullptr;
+                        stage_to_global(sbuf, lane, dst);
                     }
-                } else if (EPI == EPI_DOWN || EPI == EPI_DX) {
-                    // residual add in fp32, one rounding, scatter to the token's row
-                    uint32_t rw[16];
-                    rows_from_coalesced(sbuf, lane, ca, rw);
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        float a0, a1;
-                        unpack_bf16(rw[q], a0, a1);
-                        w[q] = pack_bf16(a0 + __uint_as_float(r[2 * q]), a1 + __uint_as_float(r[2 * q + 1]));
-                    }
-                    char *row = row_valid ? (char *)((bf16 *)p.out0 + tok * p.ldo + n) : nullptr;
-                    store_rows_64B(sbuf, lane, w, row, valid_slots);
-                } else if (EPI == EPI_DH) {
-                    uint32_t gw[16], uw[16];
-                    rows_from_coalesced(sbuf, lane, ca, gw);
-                    rows_from_coalesced(sbuf, lane, cb, uw);
-                    uint32_t w2[16];
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        float g0, g1, u0, u1, dg0, dg1, du0, du1;
-                        unpack_bf16(gw[q], g0, g1);
-                        unpack_bf16(uw[q], u0, u1);
-                        fast_swiglu_bwd(__uint_as_float(r[2 * q]), g0, u0, dg0, du0);
-                        fast_swiglu_bwd(__uint_as_float(r[2 * q + 1]), g1, u1, dg1, du1);
-                        if (!row_valid) { dg0 = dg1 = du0 = du1 = 0.0f; }
-                        w[q] = pack_bf16(dg0, dg1);
-                        w2[q] = pack_bf16(du0, du1);
-                    }
-                    const int64_t o = (int64_t)m * p.ldo + n;
-                    store_rows_64B(sbuf, lane, w, (char *)((bf16 *)p.out0 + o), valid_slots);
-                    store_rows_64B(sbuf, lane, w2, (char *)((bf16 *)p.out1 + o), valid_slots);
-                } else {   // EPI_DW: weight-gradient tile, overwrite or accumulate
+                } else {
+                    // ---- weight-gradient tile, overwrite or accumulate
+                    const int valid_slots = min(4, (n_end - n) / 8);
+                    uint32_t w[16];
                     const int64_t o = (int64_t)m * p.gldo[tl.g] + n;
                     char *row = row_valid ? (char *)p.gout[tl.g] + o * esz : nullptr;
                     if (p.out_fp32) {
@@ -898,6 +1151,7 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 }
             }
+            if (!ok) break;
             if (!zero_acc) {
                 tc_fence_before();
                 __syncwarp();
@@ -909,9 +1163,21 @@ k_umma_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+#ifdef SKIPFFN_ROLE_CYCLES
+        if (ew == 0 && lane == 0 && rank == 0) {
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 4], (int)(role_wait >> 4));
+            atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 5], (int)((clock64() - role_e0 - role_wait) >> 4));
+        }
+#endif
     }
 
     // ---------------------------------------------------------------------- teardown
+    // After a wait ran out, copies or MMAs of this CTA may still be in flight: give them time to
+    // land (bounded) before the shared and tensor memory they target is given up.
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
     tc_fence_before();
     __syncthreads();
     if (PAIR) cluster_sync_all();   // neither SM leaves while the other may still touch its memory
@@ -942,54 +1208,91 @@ static EncodeTiledFn get_encode()
 }
 
 // 2-D bf16 row-major array [outer, inner] with row pitch `pitch` elements; box = [box_outer, 64].
-// Out-of-range parts of a box read as zero.
-static bool make_map(CUtensorMap *m, const void *base, int64_t inner, int64_t outer, int64_t pitch,
-                     int box_outer)
+// Out-of-range parts of a box read as zero.  With dim2 > 0 the map has a third, outermost
+// dimension of dim2 entries `stride2_bytes` apart (which may be smaller than the row pitch: the
+// 64-column slabs of an MN-major array) and the box spans two of them.  Encoded maps are kept in
+// the caller's cache (a handle sees the same few arrays call after call), looked up by every field
+// that enters the map.
+static_assert(sizeof(CUtensorMap) == TMAP_BYTES, "tensor map size");
+static bool make_map(CUtensorMap *m, TmapCache *cache, const void *base, int64_t inner, int64_t outer,
+                     int64_t pitch, int box_outer, int64_t dim2 = 0, int64_t stride2_bytes = 0)
 {
+    if (!base) return false;
+    if (cache) {
+        for (int i = 0; i < cache->used; ++i) {
+            const TmapKey &k = cache->key[i];
+            if (k.base == base && k.inner == inner && k.outer == outer && k.pitch == pitch && k.box_outer == box_outer &&
+                k.dim2 == dim2 && k.stride2 == stride2_bytes) {
+                memcpy(m, cache->map[i], TMAP_BYTES);
+                return true;
+            }
+        }
+    }
     EncodeTiledFn enc = get_encode();
-    if (!enc || !base) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-    cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
-    cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
-    cuuint32_t es[2] = {1u, 1u};
-    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)dim2};
+    cuuint64_t strides[2] = {(cuuint64_t)pitch * 2, (cuuint64_t)stride2_bytes};
+    cuuint32_t box[3] = {64u, (cuuint32_t)box_outer, 2u};
+    cuuint32_t es[3] = {1u, 1u, 1u};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, dim2 > 0 ? 3 : 2, const_cast<void *>(base), dims, strides,
                      box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    if (r != CUDA_SUCCESS) return false;
+    if (cache) {
+        const int i = cache->used < TMAP_CACHE_ENTRIES ? cache->used++ : (cache->next++ % TMAP_CACHE_ENTRIES);
+        cache->key[i] = TmapKey{base, inner, outer, pitch, box_outer, dim2, stride2_bytes};
+        memcpy(cache->map[i], m, TMAP_BYTES);
+    }
+    return true;
 }
 
-static int g_num_sms = 0;
+// What the launch code has to know about a device, looked up once per device.
+constexpr int MAX_DEVICES = 64;
+struct DeviceInfo { int num_sms; };
+static DeviceInfo g_dev[MAX_DEVICES];
+// Process-wide switches, read from the environment once: SKIPFFN_PDL=0 launches without
+// programmatic dependent launch; SKIPFFN_SINGLE_CTA=1 selects the one-CTA-per-tile shape.
+struct Switches { int pdl, single; };
+static const Switches &switches()
+{
+    static const Switches sw = [] {
+        Switches v;
+        const char *e = getenv("SKIPFFN_PDL");
+        v.pdl = (e && atoi(e) == 0) ? 0 : 1;
+        e = getenv("SKIPFFN_SINGLE_CTA");
+        v.single = (e && atoi(e) != 0) ? 1 : 0;
+        return v;
+    }();
+    return sw;
+}
 
 // Launch one instantiation.  PAIR kernels run as clusters of two CTAs; `workers` counts tiles
 // processed concurrently (CTAs, or CTA pairs).
 template <int EPI, bool A_MN, bool B_MN, bool PAIR>
-static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
-                            const CUtensorMap &b2, const CUtensorMap &a3, const UmmaParams &p,
-                            int64_t max_tiles, cudaStream_t s)
+static cudaError_t launch_k(int dev, const TmapSet &tm, const UmmaParams &p, int64_t max_tiles, cudaStream_t s)
 {
     constexpr int SMEM = Shape<PAIR>::SMEM_BYTES;
-    static int max_workers = -1;   // -1 not yet queried; 0 unavailable
+    static int max_workers_p1[MAX_DEVICES];   // per device: 0 not yet queried, else workers + 1
     auto kern = k_umma_gemm<EPI, A_MN, B_MN, PAIR>;
-    if (max_workers < 0) {
+    if (max_workers_p1[dev] == 0) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
         if (e != cudaSuccess) return e;
+        int n = g_dev[dev].num_sms;
         if (PAIR) {
             cudaLaunchConfig_t q = {};
-            q.gridDim = dim3(2 * g_num_sms);
+            q.gridDim = dim3(2 * g_dev[dev].num_sms);
             q.blockDim = dim3(UMMA_THREADS);
             q.dynamicSmemBytes = SMEM;
             cudaLaunchAttribute at[1];
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
             q.attrs = at; q.numAttrs = 1;
-            int n = 0;
             e = cudaOccupancyMaxActiveClusters(&n, kern, &q);
             if (e != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
-            max_workers = n;
-        } else {
-            max_workers = g_num_sms;
         }
+        max_workers_p1[dev] = n + 1;
     }
+    const int max_workers = max_workers_p1[dev] - 1;
     if (max_workers <= 0) return cudaErrorNotSupported;
     // `max_tiles` = upper bound of the work items the launch can be cut into (tiles, or groups of
     // K-blocks when tiles are split along K); every worker has its own hand-over slot
@@ -1006,33 +1309,33 @@ static cudaError_t launch_k(const CUtensorMap &a, const CUtensorMap &b, const CU
     at[0].val.clusterDim.x = PAIR ? 2 : 1; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     // let this kernel's set-up overlap the tail of the previous kernel on the stream (the kernel
     // itself waits for its predecessors before it reads global memory)
-    static int pdl = -1;
-    if (pdl < 0) { const char *e = getenv("SKIPFFN_PDL"); pdl = (e && atoi(e) == 0) ? 0 : 1; }
     at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at; cfg.numAttrs = pdl ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, kern, a, b, a2, b2, a3, p);
+    cfg.attrs = at; cfg.numAttrs = switches().pdl ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, kern, tm, p);
 }
 
 template <bool PAIR>
-static cudaError_t dispatch(int epi, const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &a2,
-                            const CUtensorMap &b2, const CUtensorMap &a3, const UmmaParams &p,
-                            int64_t max_tiles, cudaStream_t s)
+static cudaError_t dispatch(int dev, int epi, const TmapSet &tm, const UmmaParams &p, int64_t max_tiles, cudaStream_t s)
 {
     switch (epi) {
-    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
-    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
-    case EPI_DH:     return launch_k<EPI_DH, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
-    case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
-    case EPI_DX:     return launch_k<EPI_DX, false, true, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
-    case EPI_PLAIN:  return launch_k<EPI_DW, false, false, PAIR>(a, b, a2, b2, a3, p, max_tiles, s);
+    case EPI_GATEUP: return launch_k<EPI_GATEUP, false, false, PAIR>(dev, tm, p, max_tiles, s);
+    case EPI_DOWN:   return launch_k<EPI_DOWN, false, false, PAIR>(dev, tm, p, max_tiles, s);
+    case EPI_DH:     return launch_k<EPI_DH, true, false, PAIR>(dev, tm, p, max_tiles, s);
+    case EPI_DW:     return launch_k<EPI_DW, true, true, PAIR>(dev, tm, p, max_tiles, s);
+    case EPI_DX:     return launch_k<EPI_DX, true, false, PAIR>(dev, tm, p, max_tiles, s);
+    case EPI_PLAIN:  return launch_k<EPI_DW, false, false, PAIR>(dev, tm, p, max_tiles, s);
     default: return cudaErrorInvalidValue;
     }
 }
 
-// GemmArgs conventions: an operand with ld_k == 1 is K-major ([outer = M or N rows, inner = K]),
-// otherwise MN-major with ld_mn == 1 ([outer = K rows, inner = M or N]).  a_outer / b_outer give the
-// number of addressable rows of each array.
+// GemmArgs conventions: C[m, n] = sum_k A(m, k) * B(n, k).  An operand with ld_k == 1 is K-major
+// ([outer = M or N rows, inner = K]), otherwise MN-major with ld_mn == 1 ([outer = K rows, inner =
+// M or N]).  a_outer / b_outer give the number of addressable rows of each array.
+// Token problems (gate/up, down, dH, dX) arrive with the WEIGHTS as A (M = weight rows) and the
+// compacted token rows as B (N = token bound, the device-resident kept count when n_from_nk);
+// their outputs and epilogue inputs are token-major arrays [token, ldo].  gate/up: A = W_gate,
+// A2 = W_up.  dX: second K segment A2 = W_up, B2 = dU.
 // `n` > 1 (weight gradients only): up to three independent problems with the same K in one launch;
 // problems 1 and 2 share their B operand.
 static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStream_t s)
@@ -1040,46 +1343,83 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     if (n < 1 || n > 3 || (n > 1 && epi != EPI_DW) || epi < 0 || epi > EPI_PLAIN) return cudaErrorInvalidValue;
     if (n == 3 && (gs[2].B != gs[1].B || gs[2].ldb_k != gs[1].ldb_k || gs[2].N != gs[1].N))
         return cudaErrorInvalidValue;
-    if (g_num_sms == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    if (g_dev[dev].num_sms == 0) {
+        e = cudaDeviceGetAttribute(&g_dev[dev].num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
     }
     const GemmArgs &g = gs[0];
     const bool gateup = epi == EPI_GATEUP;
-    CUtensorMap mA, mB, mA2, mB2, mA3;
+    const bool tok = epi != EPI_DW && epi != EPI_PLAIN;
+    TmapSet tm;
     bool ok = true;
     auto mk = [&](CUtensorMap *m, const GemmArgs &q, const void *base, bool is_a) {
         const int64_t ld_mn = is_a ? q.lda_m : q.ldb_n, ld_k = is_a ? q.lda_k : q.ldb_k;
         const int64_t outer = is_a ? q.a_outer : q.b_outer;
-        if (ld_k != 1) return make_map(m, base, is_a ? q.M : q.N, outer, ld_k, BK);   // MN-major
-        return make_map(m, base, (int64_t)q.K, outer, ld_mn, is_a ? BM : 64);          // K-major
+        if (ld_k != 1) return make_map(m, q.tmaps, base, is_a ? q.M : q.N, outer, ld_k, BK);   // MN-major
+        // K-major: A arrives in one box of 128 rows (gate/up: 64 gate + 64 up rows), B in 64-row pieces
+        return make_map(m, q.tmaps, base, (int64_t)q.K, outer, ld_mn, is_a ? (gateup ? BM / 2 : BM) : 64);
     };
-    ok &= mk(&mA, g, g.A, true);
-    ok &= mk(&mB, g, g.B, false);
+    // 3-D view of an MN-major array: [K rows][extent / 64 slabs][64 columns]; only when the slabs tile
+    // the extent exactly (a ragged last slab would reach into the next row)
+    auto mk_slabs = [&](CUtensorMap *m, const GemmArgs &q, const void *base, bool is_a) {
+        const int64_t ext = is_a ? q.M : q.N, ld_k = is_a ? q.lda_k : q.ldb_k, outer = is_a ? q.a_outer : q.b_outer;
+        if (ld_k == 1 || ext % 64 != 0) return false;
+        return make_map(m, q.tmaps, base, 64, outer, ld_k, BK, ext / 64, 128);
+    };
+    ok &= mk(&tm.A, g, g.A, true);
+    ok &= mk(&tm.B, g, g.B, false);
     if (n > 1) {
-        ok &= mk(&mA2, gs[1], gs[1].A, true);
-        ok &= mk(&mB2, gs[1], gs[1].B, false);
+        ok &= mk(&tm.A2, gs[1], gs[1].A, true);
+        ok &= mk(&tm.B2, gs[1], gs[1].B, false);
     } else {
-        if (g.A2) ok &= mk(&mA2, g, g.A2, true); else mA2 = mA;
-        if (g.B2) ok &= mk(&mB2, g, g.B2, false); else mB2 = mB;
+        if (g.A2) ok &= mk(&tm.A2, g, g.A2, true); else tm.A2 = tm.A;
+        if (g.B2) ok &= mk(&tm.B2, g, g.B2, false); else tm.B2 = tm.B;
     }
-    if (n > 2) ok &= mk(&mA3, gs[2], gs[2].A, true); else mA3 = mA;
+    if (n > 2) ok &= mk(&tm.A3, gs[2], gs[2].A, true); else tm.A3 = tm.A;
     if (!ok) return cudaErrorInvalidValue;
+    tm.Bw = tm.B; tm.B2w = tm.B2;
+    tm.A1 = tm.A; tm.A21 = tm.A2; tm.A31 = tm.A3; tm.B1 = tm.B; tm.B21 = tm.B2;
+    int a_one = 0, b_one = 0, gu_one = 0;
+    if (tok) {   // token rows (K-major B) in 128-row boxes
+        ok &= make_map(&tm.Bw, g.tmaps, g.B, (int64_t)g.K, g.b_outer, g.ldb_n, 128);
+        if (g.B2) ok &= make_map(&tm.B2w, g.tmaps, g.B2, (int64_t)g.K, g.b_outer, g.ldb_n, 128); else tm.B2w = tm.Bw;
+        if (!ok) return cudaErrorInvalidValue;
+    }
+    if (g.one_box_loads) {
+        if (gateup) {   // gate and up rows as the two entries of a third dimension
+            const char *lo = (const char *)g.A, *hi = (const char *)g.A2;
+            gu_one = 1;
+            if (hi < lo) { const char *t = lo; lo = hi; hi = t; gu_one = 2; }
+            const int64_t delta = hi - lo;
+            if (delta <= 0 || delta % 16 != 0 || delta >= ((int64_t)1 << 40) ||
+                !make_map(&tm.A1, g.tmaps, lo, (int64_t)g.K, g.a_outer, g.lda_m, BM / 2, 2, delta))
+                gu_one = 0;
+        } else if (g.lda_k != 1 && epi == EPI_DW) {
+            // (measured: for the transposed weight operand of dH / dX, streamed from HBM, one box per
+            // slab is as fast or faster; the weight-gradient operands sit in L2 and gain 6 %)
+            a_one = mk_slabs(&tm.A1, g, g.A, true) ? 1 : 0;
+            if (a_one && n > 1) a_one = mk_slabs(&tm.A21, gs[1], gs[1].A, true) ? 1 : 0;
+            if (a_one && n == 1 && g.A2) a_one = mk_slabs(&tm.A21, g, g.A2, true) ? 1 : 0;
+            if (a_one && n > 2) a_one = mk_slabs(&tm.A31, gs[2], gs[2].A, true) ? 1 : 0;
+        }
+        if (g.ldb_k != 1) {
+            b_one = mk_slabs(&tm.B1, g, g.B, false) ? 1 : 0;
+            if (b_one && n > 1) b_one = mk_slabs(&tm.B21, gs[1], gs[1].B, false) ? 1 : 0;
+        }
+    }
 
     UmmaParams p;
     p.M = g.M; p.N = g.N; p.K = g.K;
-    p.m_from_nk = g.m_from_nk; p.k_from_nk = g.k_from_nk;
+    p.n_from_nk = g.n_from_nk; p.k_from_nk = g.k_from_nk;
     p.segments = epi == EPI_DX ? 2 : 1;
+    p.force_stages = g.tune_stages > 0 ? g.tune_stages : 0;
+    // tile width override: any multiple of 16 for token problems, of 32 for the weight gradients
     p.force_bn = 0;
-    p.force_stages = 0;
-    if (const char *e = getenv("SKIPFFN_STAGES")) p.force_stages = atoi(e);
-    if (const char *e = getenv("SKIPFFN_TILE_N")) {   // tuning override: accumulator columns per tile
-        int v = atoi(e);
-        if (v >= 32 && v <= BN && v % 32 == 0) p.force_bn = v;
-    }
+    if (g.tune_tile_n >= 32 && g.tune_tile_n <= BN && g.tune_tile_n % (tok ? 16 : 32) == 0) p.force_bn = g.tune_tile_n;
     p.status = const_cast<int32_t *>(g.status);
     p.idx = g.idx;
     p.out0 = g.out0; p.out1 = g.out1; p.out2 = g.out2;
@@ -1094,37 +1434,35 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_slots = (float4 *)g.sk_slots;
     p.sk_flags = g.sk_flags;
     p.sk_epoch = g.sk_epoch;
-    // Test hook for the failure path: with SKIPFFN_TEST_LOST_HANDOVER set, units that finish a tile
-    // wait for a hand-over flag value that no producer writes, so their bounded wait runs out, the
-    // kernel records SKIPFFN_ETIMEOUT (site SITE_EPI_PARTIAL) and returns normally after about 1 s.
-    p.sk_wait_skew = 0;
-    if (const char *e = getenv("SKIPFFN_TEST_LOST_HANDOVER")) { if (atoi(e) != 0) p.sk_wait_skew = 0x40000000; }
+    p.sk_wait_skew = g.sk_wait_skew;
+    p.a_one = a_one; p.b_one = b_one; p.gu_one = gu_one;
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
     static const int sk_threshold[6] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40, /*PLAIN*/ 32};
-    p.streamk = (g.sk_slots && g.sk_flags) ? sk_threshold[epi] : 0;
-    if (const char *e = getenv("SKIPFFN_STREAMK")) { int v = atoi(e); if (v >= 0) p.streamk = v; }
+    p.streamk = (g.sk_slots && g.sk_flags) ? (g.tune_streamk >= 0 ? g.tune_streamk : sk_threshold[epi]) : 0;
 
-    // SM pairs by default; SKIPFFN_SINGLE_CTA=1 (or a device that cannot co-schedule pairs) selects
-    // the one-CTA-per-tile shape
-    static int single = -1;
-    if (single < 0) { const char *e = getenv("SKIPFFN_SINGLE_CTA"); single = (e && atoi(e) != 0) ? 1 : 0; }
-    const int n_tile = gateup ? BN / 2 : (p.force_bn > 0 ? p.force_bn : BN);   // output columns per tile
+    const int tile_w = p.force_bn > 0 ? p.force_bn : BN;   // accumulator columns per tile
     // with K splitting a tile can be shared by several workers: allow one worker per 4 K-blocks
     const int64_t kb = ((int64_t)g.K + BK - 1) / BK * p.segments;
     const int64_t per_tile = p.streamk ? (kb >= 8 ? kb / 4 : 1) : 1;
     auto max_items = [&](int tile_m) {
         int64_t t = 0;
-        for (int i = 0; i < n; ++i)
-            t += (((int64_t)gs[i].M + tile_m - 1) / tile_m) * (((int64_t)gs[i].N + n_tile - 1) / n_tile);
+        const int m_unit = gateup ? tile_m / 2 : tile_m;
+        for (int i = 0; i < n; ++i) {
+            const int64_t cols = tok ? (((int64_t)gs[i].N + 15) & ~(int64_t)15) : (int64_t)gs[i].N;
+            t += (((int64_t)gs[i].M + m_unit - 1) / m_unit) * ((cols + tile_w - 1) / tile_w);
+        }
         return t * per_tile;
     };
-    if (!single) {
-        cudaError_t e = dispatch<true>(epi, mA, mB, mA2, mB2, mA3, p, max_items(2 * BM), s);
+    // SM pairs by default; the one-CTA-per-tile shape when asked for or when the device cannot
+    // co-schedule pairs
+    static int no_pairs[MAX_DEVICES];
+    if (!switches().single && !no_pairs[dev]) {
+        e = dispatch<true>(dev, epi, tm, p, max_items(2 * BM), s);
         if (e != cudaErrorNotSupported) return e;
         (void)cudaGetLastError();
-        single = 1;
+        no_pairs[dev] = 1;
     }
-    return dispatch<false>(epi, mA, mB, mA2, mB2, mA3, p, max_items(BM), s);
+    return dispatch<false>(dev, epi, tm, p, max_items(BM), s);
 }
 
 cudaError_t launch_umma_gemm(int epi, const GemmArgs &g, cudaStream_t s)

@@ -37,7 +37,7 @@ class DeviceWorkload:
 
 
 def run(w, dense=False, path=0, grad_fp32=False, accumulate_dw=False, inplace=False, dev=None,
-        dw_init=None):
+        dw_init=None, tune=None):
     """Forward + backward through the C ABI; returns a dict of device tensors and the context."""
     import torch
     import paper_2503_21817_b200 as sk
@@ -45,6 +45,8 @@ def run(w, dense=False, path=0, grad_fp32=False, accumulate_dw=False, inplace=Fa
     dt = sk.BF16 if w.dtype == "bf16" else sk.FP32
     ctx = sk.SkipFFN(w.C, w.I, max(w.N, 1), dtype=dt, dense=dense, path=path, grad_fp32=grad_fp32,
                      accumulate_dw=accumulate_dw)
+    if tune:
+        ctx.tune(**tune)
     x = dev.x.clone()
     dout = dev.dout.clone()
     out = ctx.forward(x, dev.mask, dev.W_gate, dev.W_up, dev.W_down, out=x if inplace else None,

@@ -65,7 +65,7 @@ def _compare(w, r, ref, mask=None):
 
 
 # ------------------------------------------------------------------ a1: compaction
-@pytest.mark.parametrize("N", [1, 31, 32, 33, 1000, 4928, 16384, 16385, 50001])
+@pytest.mark.parametrize("N", [1, 15, 16, 17, 31, 32, 33, 1000, 4095, 4096, 4097, 4928, 16384, 16385, 50001, 300000])
 def test_compaction_bit_exact(N):
     import torch
     sk = _sk()
@@ -100,28 +100,48 @@ def test_multi_tile_ragged(dtype, path):
     _compare(w, run(w, path=path), _oracle_all(w))
 
 
-@pytest.mark.parametrize("tile_n", [128, 160, 192, 224, 256])
-def test_every_tile_width(tile_n, monkeypatch):
-    # tiles are 256 columns wide by default; the narrower widths the kernel supports are forced in turn
-    monkeypatch.setenv("SKIPFFN_TILE_N", str(tile_n))
+@pytest.mark.parametrize("tile_n", [32, 48, 96, 128, 160, 192, 224, 256])
+def test_every_tile_width(tile_n):
+    # tiles are 256 accumulator columns wide by default; narrower widths are forced in turn (token
+    # problems take any multiple of 16, the weight-gradient tiles multiples of 32)
     w = wl.small_case(21, "bf16", 576, 1000, 3, 20, 200, 0.6)
-    _compare(w, run(w), _oracle_all(w))
+    _compare(w, run(w, tune=dict(tile_n=tile_n)), _oracle_all(w))
+
+
+@pytest.mark.parametrize("nk", [1, 15, 16, 17, 63, 64, 65, 255, 256, 257, 300, 511, 513])
+def test_kept_counts_around_tile_and_mma_granularity(nk):
+    # the kept count decides the width of the last token tile (a multiple of 16) and the length
+    # of the last K-block of the weight-gradient reductions: every boundary case of both
+    base = wl.uniform_batch(45, "bf16", 192, 320, 1, 0, 600, 0, n_skip=600 - nk)
+    assert base.n_kept == nk
+    _compare(base, run(base), _oracle_all(base))
 
 
 @pytest.mark.parametrize("min_saving", [0, 1])
 @pytest.mark.parametrize("case", ["tiny", "ragged", "wide"])
-def test_k_split_schedule_forced_on_and_off(min_saving, case, monkeypatch):
-    # SKIPFFN_STREAMK = least K-blocks per worker that cutting the last waves along K must save:
+def test_k_split_schedule_forced_on_and_off(min_saving, case):
+    # the STREAMK knob = least K-blocks per worker that cutting the last waves along K must save:
     # 1 cuts whenever the tile count is not a multiple of the worker count (several hand-overs per
     # tile on these small shapes), 0 never cuts.  Both must match the oracle.
-    monkeypatch.setenv("SKIPFFN_STREAMK", str(min_saving))
     if case == "tiny":
         w = wl.config1(dtype="bf16")
     elif case == "ragged":
         w = wl.small_case(23, "bf16", 576, 1000, 3, 20, 200, 0.6)
     else:   # long reductions: I = 4096 gives 64 K-blocks for the down projection, 128 for dX
         w = wl.small_case(25, "bf16", 256, 4096, 2, 16, 200, 0.5)
-    _compare(w, run(w), _oracle_all(w))
+    _compare(w, run(w, tune=dict(streamk=min_saving)), _oracle_all(w))
+
+
+@pytest.mark.parametrize("one_box", [0, 1])
+def test_operand_tiles_fetched_with_one_or_two_boxes(one_box):
+    # shapes whose extents are multiples of 64, so that the one-box (3-D) operand loads apply; both
+    # ways of fetching must give the same bits
+    w = wl.small_case(27, "bf16", 512, 1024, 3, 20, 300, 0.5)
+    r = run(w, tune=dict(one_box=one_box))
+    _compare(w, r, _oracle_all(w))
+    ref = run(w, tune=dict(one_box=1 - one_box))
+    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+        assert np.array_equal(bits(r[k]), bits(ref[k])), k
 
 
 def test_contiguous_span_layout():
@@ -359,25 +379,27 @@ def test_dense_comparator_full_size():
     _full_size(wl.config2(), dense=True, rows_from_loops=False)
 
 
-def test_lost_hand_over_is_reported_and_the_context_stays_usable(monkeypatch):
-    # Failure path without a fault: with the test hook set, units that finish a K-split tile wait
-    # for a hand-over that never comes.  The wait is bounded (about 1 s): the kernel must return,
-    # skipffn_poll must report SKIPFFN_ETIMEOUT with the hand-over site, and the same handle must
-    # then produce correct results again.
+def test_lost_hand_over_is_reported_and_the_context_stays_usable():
+    # Failure path without a fault: on a debug handle the LOSE_HANDOVER knob makes the units that
+    # finish a K-split tile wait for a hand-over that never comes.  The wait is bounded (about
+    # 1 s): the kernel must return, skipffn_poll must report SKIPFFN_ETIMEOUT with the hand-over
+    # site, and the same handle must then produce correct results again.
     import time
     sk = _sk()
     w = wl.small_case(25, "bf16", 256, 4096, 2, 16, 200, 0.5)
     dev = DeviceWorkload(w)
-    ctx = sk.SkipFFN(w.C, w.I, w.N)
-    monkeypatch.setenv("SKIPFFN_STREAMK", "1")             # cut along K whenever tiles do not fill a wave
-    monkeypatch.setenv("SKIPFFN_TEST_LOST_HANDOVER", "1")
+    plain = sk.SkipFFN(w.C, w.I, w.N)
+    with pytest.raises(sk.SkipFFNError):
+        plain.tune(lose_handover=1)                        # the hook exists on debug handles only
+    ctx = sk.SkipFFN(w.C, w.I, w.N, debug=True)
+    ctx.tune(streamk=1, lose_handover=1)                   # cut along K whenever tiles do not fill a wave
     t0 = time.time()
     ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
     with pytest.raises(sk.SkipFFNError) as e:
         ctx.poll()
     assert e.value.status == 5 and "site 6" in str(e.value)
     assert time.time() - t0 < 30
-    monkeypatch.delenv("SKIPFFN_TEST_LOST_HANDOVER")
+    ctx.tune(lose_handover=0)
     out = ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
     ctx.poll()                                              # status word was cleared by the failed poll
     check(to_host(out), oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down), "bf16", "out after recovery")
