@@ -247,7 +247,8 @@ def run_ours(args):
     Wg, Wu, Wd = h_bf16(w.W_gate).to(dev), h_bf16(w.W_up).to(dev), h_bf16(w.W_down).to(dev)
     out, dx = torch.empty_like(x), torch.empty_like(x)
     dWg, dWu, dWd = torch.empty_like(Wg), torch.empty_like(Wu), torch.empty_like(Wd)
-    ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense, prenorm=args.prenorm)
+    ctx = sk.SkipFFN(C, I, N, dtype=sk.BF16, dense=args.dense, prenorm=args.prenorm, recompute=args.recompute,
+                     max_kept=None if (args.dense or not args.kept_sized) else nk)
     if args.tune:       # launch knobs of the handle (skipffn_tune), e.g. --tune one_box=0,streamk=0
         ctx.tune(**{k: int(v) for k, v in (kv.split("=") for kv in args.tune.split(","))})
     if args.dense:
@@ -421,6 +422,26 @@ def run_ours(args):
             "frac_of_burst_bf16_peak": tf_s / pk["bf16_tflops"], "clocks": clocks_sus,
             "mcycles_per_step": ms_s * clocks_sus["sm_mhz"] * 1e-3 if clocks_sus.get("sm_mhz") else None,
             "kernels": sus_kernels}
+        # memory modes: bytes a handle holds between forward and backward (saved) and inside a call
+        # (scratch, shareable between layers), and the time of the recomputing mode
+        def sizes(**kw):
+            c = sk.SkipFFN(C, I, N, **kw)
+            return {"saved_bytes": c.saved_bytes, "scratch_bytes": c.scratch_bytes}
+        rc = sk.SkipFFN(C, I, N, recompute=True, max_kept=nk)
+
+        def step_rc():
+            rc.forward(x, mask, Wg, Wu, Wd, out=out)
+            rc.backward(dout, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+        for _ in range(3):
+            step_rc()
+        ms_def, _, _ = timed(step, args.steps)          # the default mode again, same thermal state
+        ms_rc, _, _ = timed(step_rc, args.steps)
+        rc.poll()
+        extras["memory_modes"] = {
+            "token_sized": sizes(), "kept_sized": sizes(max_kept=nk),
+            "kept_sized_recompute": {"saved_bytes": rc.saved_bytes, "scratch_bytes": rc.scratch_bytes,
+                                     "ms_per_step": ms_rc / args.steps, "time_vs_default": ms_rc / ms_def}}
+        del rc
         # the other single-GPU workloads, same weights
         dbuf.clear()
         weights_host = (w.W_gate, w.W_up, w.W_down)
@@ -744,6 +765,9 @@ def main():
     ap.add_argument("--dense", action="store_true", help="in-library dense comparator (mask ignored)")
     ap.add_argument("--prenorm", action="store_true",
                     help="pre-norm variant: out = x + FFN(RMSNorm(x) * gamma), with dgamma in the backward")
+    ap.add_argument("--recompute", action="store_true",
+                    help="memory mode: the forward keeps no G, U, H, the backward runs the gate/up GEMM again")
+    ap.add_argument("--kept-sized", action="store_true", help="size the compacted arrays by the workload's kept count")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-sample-tokens", type=int, default=24)
     ap.add_argument("--no-cpu-baseline", action="store_true")

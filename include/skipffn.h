@@ -37,7 +37,8 @@ typedef enum {
     SKIPFFN_OK = 0,
     SKIPFFN_EINVAL = 1,       /* null pointer, bad shape, misaligned pointer, forward missing */
     SKIPFFN_EUNSUPPORTED = 2, /* shape outside what the kernels handle */
-    SKIPFFN_EWORKSPACE = 3,   /* workspace too small for max_tokens */
+    SKIPFFN_EWORKSPACE = 3,   /* workspace too small for max_tokens / max_kept; reported by skipffn_poll
+                                 when a mask kept more than max_kept tokens */
     SKIPFFN_ECUDA = 4,        /* a CUDA runtime / driver call failed */
     SKIPFFN_ETIMEOUT = 5      /* a device-side wait hit its limit (reported by skipffn_poll) */
 } skipffn_status;
@@ -58,6 +59,7 @@ typedef struct {
     int32_t path;            /* skipffn_path */
     int32_t prenorm;         /* 1: pre-norm variant (skipffn_forward_prenorm / _backward_prenorm) */
     int32_t debug;           /* 1: debug handle: extra device-side checks (see skipffn_poll), test hooks */
+    int32_t recompute;       /* 1: the forward keeps no G, U, H; the backward computes them again */
 } skipffn_config;
 
 /* Host-side handle linking one forward call to its backward call.  It points into the caller's
@@ -65,11 +67,38 @@ typedef struct {
  * intermediates G, U, H (and dG, dU during backward) live. */
 typedef struct skipffn_saved skipffn_saved;
 
-/* Bytes of device workspace needed for up to max_tokens tokens (0 if cfg is invalid). */
+/* Device memory of a handle.  It has two parts:
+ *   saved    what must survive from a forward call to its backward call: the kept-row list, the kept
+ *            rows of x and -- unless cfg.recompute -- the SwiGLU intermediates G, U, H;
+ *   scratch  what only lives inside one call (dG, dU, the kept rows of dout, K-split hand-over slots,
+ *            and G, U, H of a recomputing handle).  Handles whose calls never overlap on the GPU (the
+ *            layers of one model, run one after the other) may share one scratch buffer.
+ * max_tokens bounds B*S of any call; max_kept (<= max_tokens) bounds the number of kept tokens and
+ * sizes every compacted array, so a model that skips 75 % of its visual tokens does not pay for the
+ * rows it never sends through the FFN.  A mask that keeps more than max_kept tokens is not an
+ * out-of-bounds access: the first max_kept kept tokens take the FFN, the others are treated as
+ * skipped, and skipffn_poll reports SKIPFFN_EWORKSPACE.
+ * Recompute mode trades time for memory (the idea of not storing what the backward can rebuild):
+ * the forward stores only H, transiently, for the down projection; the backward runs the gate/up
+ * GEMM again (one more launch, +4 Nk C I flops).  Results are the same bits in both modes.
+ * All sizes are 0 if the arguments are invalid; buffers must be 1024-byte aligned. */
+size_t skipffn_saved_bytes(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept);
+size_t skipffn_scratch_bytes(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept);
+/* saved + scratch in one buffer */
+size_t skipffn_workspace_bytes_kept(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept);
+/* the same with max_kept = max_tokens */
 size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens);
 
-/* Create a handle over `workspace` (device memory, 1024-byte aligned, workspace_bytes long).
- * Host-only: nothing is launched.  EWORKSPACE if the buffer is too small. */
+/* Create a handle.  Host-only: nothing is launched.  EWORKSPACE if a buffer is too small.
+ *   skipffn_saved_create_split : separate saved and scratch buffers;
+ *   skipffn_saved_create_kept  : one buffer of skipffn_workspace_bytes_kept bytes;
+ *   skipffn_saved_create       : one buffer of skipffn_workspace_bytes bytes (max_kept = max_tokens). */
+skipffn_status skipffn_saved_create_split(skipffn_saved **saved, const skipffn_config *cfg,
+                                          void *saved_mem, size_t saved_bytes, void *scratch_mem,
+                                          size_t scratch_bytes, int64_t max_tokens, int64_t max_kept);
+skipffn_status skipffn_saved_create_kept(skipffn_saved **saved, const skipffn_config *cfg,
+                                         void *workspace, size_t workspace_bytes, int64_t max_tokens,
+                                         int64_t max_kept);
 skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg,
                                     void *workspace, size_t workspace_bytes, int64_t max_tokens);
 void skipffn_saved_destroy(skipffn_saved *saved);
@@ -221,8 +250,9 @@ skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_ou
  * 2 gate/up GEMM, 3 down GEMM, 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate, 8 dW_up,
  * 9 dX GEMM.  The tensor-core path computes the requested weight gradients in ONE grouped launch,
  * whose time is reported in the slot of the first of them (6 when dW_down is requested) with the
- * other two slots 0.  Slot 10 (pre-norm variant): the normalisation's backward (dx rows and dgamma). */
-#define SKIPFFN_PROFILE_SLOTS 11
+ * other two slots 0.  Slot 10 (pre-norm variant): the normalisation's backward (dx rows and dgamma).
+ * Slot 11 (recomputing handles): the gate/up GEMM run again at the start of the backward. */
+#define SKIPFFN_PROFILE_SLOTS 12
 skipffn_status skipffn_profile_enable(skipffn_saved *saved, int32_t on);
 skipffn_status skipffn_profile_read(skipffn_saved *saved, float *ms);
 

@@ -20,12 +20,13 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_compact_static", "skipffn_schedule_segment", "skipffn_kv_compact",
            "skipffn_forward_prenorm", "skipffn_backward_prenorm", "skipffn_summary_scratch_bytes",
            "skipffn_summary_forward", "skipffn_summary_backward", "skipffn_token_merge_scratch_bytes",
-           "skipffn_token_merge", "skipffn_tune"]
+           "skipffn_token_merge", "skipffn_tune", "skipffn_saved_bytes", "skipffn_scratch_bytes",
+           "skipffn_workspace_bytes_kept", "skipffn_saved_create_kept", "skipffn_saved_create_split"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4}
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
-                 "dw_up", "dx", "norm_bwd"]
+                 "dw_up", "dx", "norm_bwd", "recompute"]
 
 
 class SkipFFNError(RuntimeError):
@@ -38,7 +39,7 @@ class _Config(ctypes.Structure):
     _fields_ = [("C", ctypes.c_int32), ("I", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("dense", ctypes.c_int32), ("grad_dtype_fp32", ctypes.c_int32),
                 ("accumulate_dw", ctypes.c_int32), ("path", ctypes.c_int32),
-                ("prenorm", ctypes.c_int32), ("debug", ctypes.c_int32)]
+                ("prenorm", ctypes.c_int32), ("debug", ctypes.c_int32), ("recompute", ctypes.c_int32)]
 
 
 def load_library() -> ctypes.CDLL:
@@ -56,6 +57,13 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_workspace_bytes.argtypes = [cfgp, i64]
     lib.skipffn_saved_create.restype = i32
     lib.skipffn_saved_create.argtypes = [ctypes.POINTER(vp), cfgp, vp, ctypes.c_size_t, i64]
+    for fn in (lib.skipffn_saved_bytes, lib.skipffn_scratch_bytes, lib.skipffn_workspace_bytes_kept):
+        fn.restype = ctypes.c_size_t
+        fn.argtypes = [cfgp, i64, i64]
+    lib.skipffn_saved_create_kept.restype = i32
+    lib.skipffn_saved_create_kept.argtypes = [ctypes.POINTER(vp), cfgp, vp, ctypes.c_size_t, i64, i64]
+    lib.skipffn_saved_create_split.restype = i32
+    lib.skipffn_saved_create_split.argtypes = [ctypes.POINTER(vp), cfgp, vp, ctypes.c_size_t, vp, ctypes.c_size_t, i64, i64]
     lib.skipffn_saved_destroy.restype = None
     lib.skipffn_saved_destroy.argtypes = [vp]
     lib.skipffn_plan.restype = i32
@@ -108,9 +116,9 @@ def load_library() -> ctypes.CDLL:
 
 
 def _cfg(C, I, dtype=BF16, dense=False, grad_fp32=False, accumulate_dw=False, path=PATH_DEFAULT,
-         prenorm=False, debug=False):
+         prenorm=False, debug=False, recompute=False):
     return _Config(int(C), int(I), int(dtype), int(bool(dense)), int(bool(grad_fp32)),
-                   int(bool(accumulate_dw)), int(path), int(bool(prenorm)), int(bool(debug)))
+                   int(bool(accumulate_dw)), int(path), int(bool(prenorm)), int(bool(debug)), int(bool(recompute)))
 
 
 def skipffn_workspace_bytes(C, I, max_tokens, dtype=BF16) -> int:
@@ -246,28 +254,46 @@ class SkipFFN:
 
     def __init__(self, C: int, I: int, max_tokens: int, dtype: int = BF16, dense: bool = False,
                  grad_fp32: bool = False, accumulate_dw: bool = False, path: int = PATH_DEFAULT,
-                 device="cuda", prenorm: bool = False, debug: bool = False):
+                 device="cuda", prenorm: bool = False, debug: bool = False, recompute: bool = False,
+                 max_kept=None, scratch_from=None):
+        """``max_kept`` bounds the kept tokens of any call (default: ``max_tokens``) and sizes the
+        compacted arrays.  ``recompute``: the forward keeps no G, U, H.  ``scratch_from``: another
+        context of the same configuration whose scratch buffer this one shares (calls of the two
+        must not overlap on the GPU)."""
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("Skip-FFN needs a CUDA device (sm_100a); there is no CPU path")
         self._torch = torch
         self.lib = load_library()
         self.C, self.I, self.dtype, self.max_tokens = int(C), int(I), int(dtype), int(max_tokens)
+        self.max_kept = self.max_tokens if max_kept is None else int(max_kept)
         self.grad_fp32 = bool(grad_fp32) or dtype == FP32
         self.prenorm = bool(prenorm)
-        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path, prenorm, debug)
+        self.cfg = _cfg(C, I, dtype, dense, grad_fp32, accumulate_dw, path, prenorm, debug, recompute)
         self.device = torch.device(device)
-        nbytes = int(self.lib.skipffn_workspace_bytes(ctypes.byref(self.cfg), self.max_tokens))
-        if nbytes == 0:
-            raise SkipFFNError(1, "skipffn_workspace_bytes")
-        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=self.device)
-        base = self.workspace.data_ptr()
-        self._ws_ptr = (base + 1023) // 1024 * 1024
+        cfgp = ctypes.byref(self.cfg)
+        self.saved_bytes = int(self.lib.skipffn_saved_bytes(cfgp, self.max_tokens, self.max_kept))
+        self.scratch_bytes = int(self.lib.skipffn_scratch_bytes(cfgp, self.max_tokens, self.max_kept))
+        if self.saved_bytes == 0:
+            raise SkipFFNError(1, "skipffn_saved_bytes")
+
+        def aligned(t):
+            return (t.data_ptr() + 1023) // 1024 * 1024
+        self.workspace = torch.empty(self.saved_bytes + 1024, dtype=torch.uint8, device=self.device)
+        if scratch_from is not None:
+            if scratch_from.scratch_bytes < self.scratch_bytes:
+                raise ValueError("the shared scratch buffer is too small for this context")
+            self.scratch = scratch_from.scratch
+        else:
+            self.scratch = torch.empty(self.scratch_bytes + 1024, dtype=torch.uint8, device=self.device)
+        self._ws_ptr = aligned(self.workspace)
         self._saved = ctypes.c_void_p()
-        st = self.lib.skipffn_saved_create(ctypes.byref(self._saved), ctypes.byref(self.cfg),
-                                           ctypes.c_void_p(self._ws_ptr), nbytes, self.max_tokens)
+        st = self.lib.skipffn_saved_create_split(ctypes.byref(self._saved), cfgp, ctypes.c_void_p(self._ws_ptr),
+                                                 self.saved_bytes, ctypes.c_void_p(aligned(self.scratch)),
+                                                 self.scratch.numel() - (aligned(self.scratch) - self.scratch.data_ptr()),
+                                                 self.max_tokens, self.max_kept)
         if st != 0:
-            raise SkipFFNError(st, "skipffn_saved_create")
+            raise SkipFFNError(st, "skipffn_saved_create_split")
         self._keep = []   # tensors the handle borrows between forward and backward
         self._shape = None
 
@@ -454,11 +480,14 @@ class SkipFFN:
         return self._view(p.value, rows * cols, self.torch_dtype).view(rows, cols).clone()
 
     def _view(self, ptr, numel, dtype):
-        """Tensor view of `numel` elements of the workspace starting at device address `ptr`."""
+        """Tensor view of `numel` elements of the handle's memory starting at device address `ptr`."""
         torch = self._torch
-        off = ptr - self.workspace.data_ptr()
         nbytes = numel * torch.empty(0, dtype=dtype).element_size()
-        return self.workspace[off:off + nbytes].view(dtype)
+        for buf in (self.workspace, self.scratch):
+            off = ptr - buf.data_ptr()
+            if 0 <= off and off + nbytes <= buf.numel():
+                return buf[off:off + nbytes].view(dtype)
+        raise ValueError("address outside the handle's buffers")
 
     def profile(self, step_fn, steps: int):
         """Run ``step_fn`` ``steps`` times with CUDA events around every kernel launch; returns the

@@ -9,7 +9,8 @@ using namespace skipffn;
 
 struct skipffn_saved {
     skipffn_config cfg;
-    int64_t max_tokens, cap;
+    int64_t max_tokens, cap;   // cap: rows of the token-indexed arrays (idx, pos)
+    int64_t max_kept, cap_k;   // cap_k: rows of the compacted arrays (kept rows only)
     size_t ws_bytes;
     int esize;
     // workspace carve-up (device)
@@ -35,40 +36,57 @@ struct skipffn_saved {
 
 namespace {
 
+// Two regions.  `saved` must survive from a forward call to its backward call; `scratch` only lives
+// inside one call, so several handles (the layers of a model) may share one scratch buffer as long
+// as their calls do not overlap.  With cfg.recompute the SwiGLU intermediates G, U, H move from the
+// saved region to the scratch region: the backward pass computes them again.
 struct Layout {
-    size_t status, idx, pos, sk_slots, Xk, dOk, G, U, H, dG, dU, Xn, rstd, dY, dg_part, total;
+    size_t status, idx, pos, Xk, Xn, rstd, saved_total;                  // saved region
+    size_t sk_slots, dOk, dG, dU, dY, dg_part, scratch_total;              // scratch region
+    size_t G, U, H;                                                        // in saved, or in scratch when recomputing
 };
 
 bool valid_cfg(const skipffn_config *c)
 {
     return c && c->C > 0 && c->I > 0 && (c->dtype == SKIPFFN_BF16 || c->dtype == SKIPFFN_FP32) &&
            (c->path == SKIPFFN_PATH_DEFAULT || c->path == SKIPFFN_PATH_SIMT) &&
-           (c->prenorm == 0 || c->prenorm == 1) && (c->debug == 0 || c->debug == 1);
+           (c->prenorm == 0 || c->prenorm == 1) && (c->debug == 0 || c->debug == 1) &&
+           (c->recompute == 0 || c->recompute == 1);
 }
 
-Layout make_layout(const skipffn_config *c, int64_t max_tokens)
+Layout make_layout(const skipffn_config *c, int64_t max_tokens, int64_t max_kept)
 {
     Layout l;
     const int64_t cap = round_up(max_tokens > 0 ? max_tokens : 1, ROW_PAD);
+    const int64_t cap_k = round_up(max_kept > 0 ? max_kept : 1, ROW_PAD);
     const size_t es = c->dtype == SKIPFFN_BF16 ? 2 : 4;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
     l.status = take((ST_WORDS + SK_FLAG_WORDS) * 4);   // status block, then the hand-over flags
     l.idx = take((size_t)cap * 4);
     l.pos = take((size_t)cap * 4);
+    l.Xk = take((size_t)cap_k * c->C * es);
+    l.Xn = take(c->prenorm ? (size_t)cap_k * c->C * es : 0);
+    l.rstd = take(c->prenorm ? (size_t)cap_k * 4 : 0);
+    if (!c->recompute) {
+        l.G = take((size_t)cap_k * c->I * es);
+        l.U = take((size_t)cap_k * c->I * es);
+        l.H = take((size_t)cap_k * c->I * es);
+    }
+    l.saved_total = off;
+    off = 0;
     l.sk_slots = take(c->dtype == SKIPFFN_BF16 ? (size_t)SK_MAX_CTAS * SK_SLOT_BYTES : 0);
-    l.Xk = take((size_t)cap * c->C * es);
-    l.dOk = take((size_t)cap * c->C * es);
-    l.G = take((size_t)cap * c->I * es);
-    l.U = take((size_t)cap * c->I * es);
-    l.H = take((size_t)cap * c->I * es);
-    l.dG = take((size_t)cap * c->I * es);
-    l.dU = take((size_t)cap * c->I * es);
-    l.Xn = take(c->prenorm ? (size_t)cap * c->C * es : 0);
-    l.rstd = take(c->prenorm ? (size_t)cap * 4 : 0);
-    l.dY = take(c->prenorm ? (size_t)cap * c->C * 4 : 0);
+    l.dOk = take((size_t)cap_k * c->C * es);
+    l.dG = take((size_t)cap_k * c->I * es);
+    l.dU = take((size_t)cap_k * c->I * es);
+    l.dY = take(c->prenorm ? (size_t)cap_k * c->C * 4 : 0);
     l.dg_part = take(c->prenorm ? (size_t)DG_CHUNKS * c->C * 4 : 0);
-    l.total = off;
+    if (c->recompute) {
+        l.G = take((size_t)cap_k * c->I * es);
+        l.U = take((size_t)cap_k * c->I * es);
+        l.H = take((size_t)cap_k * c->I * es);
+    }
+    l.scratch_total = off;
     return l;
 }
 
@@ -81,14 +99,15 @@ bool use_umma(const skipffn_saved *s)
 
 // Launch slots (also the order of skipffn_profile_read): forward 0 compaction, 1 routing of x,
 // 2 gate/up GEMM, 3 down GEMM; backward 4 routing of dout, 5 dH GEMM, 6 dW_down, 7 dW_gate,
-// 8 dW_up, 9 dX GEMM.
+// 8 dW_up, 9 dX GEMM; 10 normalisation backward (pre-norm variant); 11 the gate/up GEMM run again
+// by a recomputing handle's backward.
 enum : int { SLOT_COMPACT = 0, SLOT_ROUTE_X, SLOT_GATEUP, SLOT_DOWN, SLOT_ROUTE_DOUT, SLOT_DH,
-             SLOT_DW_DOWN, SLOT_DW_GATE, SLOT_DW_UP, SLOT_DX, SLOT_NORM_BWD };
+             SLOT_DW_DOWN, SLOT_DW_GATE, SLOT_DW_UP, SLOT_DX, SLOT_NORM_BWD, SLOT_RECOMPUTE };
 
 template <typename F>
 cudaError_t timed_launch(skipffn_saved *s, int slot, cudaStream_t st, F &&launch)
 {
-    s->launches[slot >= SLOT_ROUTE_DOUT ? 1 : 0]++;
+    s->launches[(slot >= SLOT_ROUTE_DOUT) ? 1 : 0]++;
     if (!s->profiling) return launch();
     cudaError_t e = cudaEventRecord(s->ev[2 * slot], st);
     if (e != cudaSuccess) return e;
@@ -132,7 +151,7 @@ skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int whi
     (void)which;
     if (N > 0) {
         if (timed_launch(s, SLOT_COMPACT, st, [&] {
-                return launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, st);
+                return launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, s->max_kept, st);
             }) != cudaSuccess)
             return SKIPFFN_ECUDA;
     } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
@@ -146,46 +165,89 @@ skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int whi
 
 extern "C" {
 
-size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens)
+size_t skipffn_saved_bytes(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept)
 {
-    if (!valid_cfg(cfg) || max_tokens < 0) return 0;
-    return make_layout(cfg, max_tokens).total;
+    if (!valid_cfg(cfg) || max_tokens < 0 || max_kept < 0 || max_kept > max_tokens) return 0;
+    return make_layout(cfg, max_tokens, max_kept).saved_total;
 }
 
-skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg, void *workspace,
-                                    size_t workspace_bytes, int64_t max_tokens)
+size_t skipffn_scratch_bytes(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept)
+{
+    if (!valid_cfg(cfg) || max_tokens < 0 || max_kept < 0 || max_kept > max_tokens) return 0;
+    return make_layout(cfg, max_tokens, max_kept).scratch_total;
+}
+
+size_t skipffn_workspace_bytes_kept(const skipffn_config *cfg, int64_t max_tokens, int64_t max_kept)
+{
+    if (!valid_cfg(cfg) || max_tokens < 0 || max_kept < 0 || max_kept > max_tokens) return 0;
+    const Layout l = make_layout(cfg, max_tokens, max_kept);
+    return l.saved_total + l.scratch_total;
+}
+
+size_t skipffn_workspace_bytes(const skipffn_config *cfg, int64_t max_tokens)
+{
+    return skipffn_workspace_bytes_kept(cfg, max_tokens, max_tokens);
+}
+
+skipffn_status skipffn_saved_create_split(skipffn_saved **saved, const skipffn_config *cfg, void *saved_mem,
+                                          size_t saved_bytes, void *scratch_mem, size_t scratch_bytes,
+                                          int64_t max_tokens, int64_t max_kept)
 {
     if (!saved) return SKIPFFN_EINVAL;
     *saved = nullptr;
-    if (!valid_cfg(cfg) || !workspace || max_tokens < 0) return SKIPFFN_EINVAL;
+    if (!valid_cfg(cfg) || !saved_mem || !scratch_mem || max_tokens < 0 || max_kept < 0 || max_kept > max_tokens)
+        return SKIPFFN_EINVAL;
     if ((cfg->C % 8) || (cfg->I % 8)) return SKIPFFN_EUNSUPPORTED;
     if (max_tokens > (int64_t)1 << 30) return SKIPFFN_EUNSUPPORTED;
-    if ((uintptr_t)workspace & 1023u) return SKIPFFN_EINVAL;
-    Layout l = make_layout(cfg, max_tokens);
-    if (workspace_bytes < l.total) return SKIPFFN_EWORKSPACE;
+    if (((uintptr_t)saved_mem & 1023u) || ((uintptr_t)scratch_mem & 1023u)) return SKIPFFN_EINVAL;
+    Layout l = make_layout(cfg, max_tokens, max_kept);
+    if (saved_bytes < l.saved_total || scratch_bytes < l.scratch_total) return SKIPFFN_EWORKSPACE;
     skipffn_saved *s = new (std::nothrow) skipffn_saved;
     if (!s) return SKIPFFN_EINVAL;
     memset(s, 0, sizeof(*s));
     s->cfg = *cfg;
     s->max_tokens = max_tokens;
     s->cap = round_up(max_tokens > 0 ? max_tokens : 1, ROW_PAD);
-    s->ws_bytes = workspace_bytes;
+    s->max_kept = max_kept;
+    s->cap_k = round_up(max_kept > 0 ? max_kept : 1, ROW_PAD);
+    s->ws_bytes = saved_bytes + scratch_bytes;
     s->esize = cfg->dtype == SKIPFFN_BF16 ? 2 : 4;
-    char *w = (char *)workspace;
+    char *w = (char *)saved_mem, *x = (char *)scratch_mem;
+    char *gu = cfg->recompute ? x : w;
     s->status = (int32_t *)(w + l.status);
     s->sk_flags = s->status + ST_WORDS;
-    s->sk_slots = w + l.sk_slots;
     s->idx = (int32_t *)(w + l.idx);
     s->pos = (int32_t *)(w + l.pos);
-    s->Xk = w + l.Xk; s->dOk = w + l.dOk;
-    s->G = w + l.G; s->U = w + l.U; s->H = w + l.H; s->dG = w + l.dG; s->dU = w + l.dU;
-    s->Xn = w + l.Xn; s->rstd = (float *)(w + l.rstd); s->dY = (float *)(w + l.dY);
-    s->dg_part = (float *)(w + l.dg_part);
+    s->Xk = w + l.Xk;
+    s->Xn = w + l.Xn; s->rstd = (float *)(w + l.rstd);
+    s->G = gu + l.G; s->U = gu + l.U; s->H = gu + l.H;
+    s->sk_slots = x + l.sk_slots;
+    s->dOk = x + l.dOk; s->dG = x + l.dG; s->dU = x + l.dU;
+    s->dY = (float *)(x + l.dY);
+    s->dg_part = (float *)(x + l.dg_part);
     s->planned_N = -1;
     s->tune[SKIPFFN_TUNE_STREAMK] = -1;
     s->tune[SKIPFFN_TUNE_ONE_BOX] = 1;
     *saved = s;
     return SKIPFFN_OK;
+}
+
+skipffn_status skipffn_saved_create_kept(skipffn_saved **saved, const skipffn_config *cfg, void *workspace,
+                                         size_t workspace_bytes, int64_t max_tokens, int64_t max_kept)
+{
+    if (!saved) return SKIPFFN_EINVAL;
+    *saved = nullptr;
+    if (!valid_cfg(cfg) || !workspace || max_tokens < 0 || max_kept < 0 || max_kept > max_tokens) return SKIPFFN_EINVAL;
+    const Layout l = make_layout(cfg, max_tokens, max_kept);
+    if (workspace_bytes < l.saved_total + l.scratch_total) return SKIPFFN_EWORKSPACE;
+    return skipffn_saved_create_split(saved, cfg, workspace, l.saved_total, (char *)workspace + l.saved_total,
+                                      workspace_bytes - l.saved_total, max_tokens, max_kept);
+}
+
+skipffn_status skipffn_saved_create(skipffn_saved **saved, const skipffn_config *cfg, void *workspace,
+                                    size_t workspace_bytes, int64_t max_tokens)
+{
+    return skipffn_saved_create_kept(saved, cfg, workspace, workspace_bytes, max_tokens, max_tokens);
 }
 
 skipffn_status skipffn_tune(skipffn_saved *s, int32_t what, int32_t value)
@@ -248,6 +310,28 @@ skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t 
     return do_plan(s, skip_mask, N, 0, st);
 }
 
+// G = X Wg^T, U = X Wu^T, H = silu(G) * U, with X = the kept rows (normalised in the pre-norm
+// variant).  The tensor-core kernels take the weights as the A operand (weight rows along the
+// accumulator rows) and the token rows as B; the plain-FMA kernels the other way round.
+// `store_gu` = 0 writes H only.
+static cudaError_t gate_up(skipffn_saved *s, int slot, int32_t NB, bool store_gu, cudaStream_t st)
+{
+    const int C = s->cfg.C, I = s->cfg.I;
+    const void *Xrows = s->cfg.prenorm ? s->Xn : s->Xk;
+    GemmArgs g = base_args(s);
+    if (use_umma(s)) {
+        g.A = s->Wg; g.A2 = s->Wu; g.lda_m = C; g.lda_k = 1; g.a_outer = I;
+        g.B = Xrows; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap_k;
+        g.M = I; g.N = NB; g.n_from_nk = 1; g.K = C;
+    } else {
+        g.A = Xrows; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap_k;
+        g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
+        g.M = NB; g.m_from_nk = 1; g.N = I; g.K = C;
+    }
+    g.out0 = store_gu ? s->G : nullptr; g.out1 = store_gu ? s->U : nullptr; g.out2 = s->H; g.ldo = I;
+    return run_gemm(s, slot, EPI_GATEUP, g, st);
+}
+
 static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_t *skip_mask, int64_t B,
                                    int64_t S, const int32_t *cu_seqlens, int32_t n_seq,
                                    const void *gamma, float eps, const void *W_gate, const void *W_up,
@@ -291,34 +375,21 @@ static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_
         }) != cudaSuccess)
         return SKIPFFN_ECUDA;
 
-    // G = X Wg^T, U = X Wu^T, H = silu(G) * U, with X = the kept rows (normalised in the pre-norm
-    // variant).  The tensor-core kernels take the weights as the A operand (weight rows along the
-    // accumulator rows) and the token rows as B; the plain-FMA kernels the other way round.
-    const void *Xrows = gamma ? s->Xn : s->Xk;
+    const int32_t NB = (int32_t)(N < s->max_kept ? N : s->max_kept);   // host bound of the kept count
     const bool tc = use_umma(s);
-    GemmArgs g = base_args(s);
-    if (tc) {
-        g.A = W_gate; g.A2 = W_up; g.lda_m = C; g.lda_k = 1; g.a_outer = I;
-        g.B = Xrows; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap;
-        g.M = I; g.N = (int32_t)N; g.n_from_nk = 1; g.K = C;
-    } else {
-        g.A = Xrows; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
-        g.B = W_gate; g.B2 = W_up; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
-        g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
-    }
-    g.out0 = s->G; g.out1 = s->U; g.out2 = s->H; g.ldo = I;
-    if (run_gemm(s, SLOT_GATEUP, EPI_GATEUP, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    // a recomputing handle keeps only H (for the down projection); its backward computes G, U, H again
+    if (gate_up(s, SLOT_GATEUP, NB, !s->cfg.recompute, st) != cudaSuccess) return SKIPFFN_ECUDA;
 
     // out[idx[r]] = Xk[r] + H Wd^T
-    g = base_args(s);
+    GemmArgs g = base_args(s);
     if (tc) {
         g.A = W_down; g.lda_m = I; g.lda_k = 1; g.a_outer = C;
-        g.B = s->H; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap;
-        g.M = C; g.N = (int32_t)N; g.n_from_nk = 1; g.K = I;
+        g.B = s->H; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap_k;
+        g.M = C; g.N = NB; g.n_from_nk = 1; g.K = I;
     } else {
-        g.A = s->H; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+        g.A = s->H; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap_k;
         g.B = W_down; g.ldb_n = I; g.ldb_k = 1; g.b_outer = C;
-        g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+        g.M = NB; g.m_from_nk = 1; g.N = C; g.K = I;
     }
     g.in0 = s->Xk; g.out0 = out; g.ldo = C;
     if (run_gemm(s, SLOT_DOWN, EPI_DOWN, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
@@ -359,6 +430,7 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
     s->launches[1] = 0;
     GemmArgs g;
     const bool tc = use_umma(s);
+    const int32_t NB = (int32_t)(N < s->max_kept ? N : s->max_kept);   // host bound of the kept count
 
     if (N > 0) {
         RouteArgs r;
@@ -367,16 +439,19 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
         if (timed_launch(s, SLOT_ROUTE_DOUT, st, [&] { return launch_route(r, st); }) != cudaSuccess)
             return SKIPFFN_ECUDA;
 
+        // a recomputing handle kept no G, U, H: compute them again from the kept rows
+        if (s->cfg.recompute && gate_up(s, SLOT_RECOMPUTE, NB, true, st) != cudaSuccess) return SKIPFFN_ECUDA;
+
         // dH = dOk Wd ; dG, dU through the activation
         g = base_args(s);
         if (tc) {   // dH^T[i, t] = sum_c Wd[c, i] dOk[t, c]
             g.A = s->Wd; g.lda_m = 1; g.lda_k = I; g.a_outer = C;
-            g.B = s->dOk; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap;
-            g.M = I; g.N = (int32_t)N; g.n_from_nk = 1; g.K = C;
+            g.B = s->dOk; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap_k;
+            g.M = I; g.N = NB; g.n_from_nk = 1; g.K = C;
         } else {
-            g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap;
+            g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap_k;
             g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;
-            g.M = (int32_t)N; g.m_from_nk = 1; g.N = I; g.K = C;
+            g.M = NB; g.m_from_nk = 1; g.N = I; g.K = C;
         }
         g.in0 = s->G; g.in1 = s->U; g.out0 = s->dG; g.out1 = s->dU; g.ldo = I;
         if (run_gemm(s, SLOT_DH, EPI_DH, g, st) != cudaSuccess) return SKIPFFN_ECUDA;
@@ -386,7 +461,7 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
 
     // weight gradients: reductions over the kept-token axis (K = Nk, read on the device)
     //   dWd[c, i] = sum_r dOk[r, c] H[r, i];  dWg[i, c] = sum_r dG[r, i] Xk[r, c];  dWu likewise with dU
-    const int32_t kmax = (int32_t)N;
+    const int32_t kmax = NB;
     GemmArgs dw[3];
     int dw_slot[3], n_dw = 0;
     void *dw_dst[3] = {dW_down, dW_gate, dW_up};
@@ -400,7 +475,7 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
             q.A = w == 1 ? s->dG : s->dU; q.lda_k = I; q.B = prenorm ? s->Xn : s->Xk; q.ldb_k = C;
             q.M = I; q.N = C; q.ldo = C;
         }
-        q.lda_m = 1; q.ldb_n = 1; q.a_outer = s->cap; q.b_outer = s->cap;
+        q.lda_m = 1; q.ldb_n = 1; q.a_outer = s->cap_k; q.b_outer = s->cap_k;
         q.K = kmax; q.k_from_nk = 1;
         q.out0 = dw_dst[w]; q.accumulate = s->cfg.accumulate_dw;
         q.out_fp32 = s->cfg.grad_dtype_fp32 || s->cfg.dtype == SKIPFFN_FP32;
@@ -422,12 +497,12 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
         g = base_args(s);
         if (tc) {   // dx^T[c, t] = sum_i Wg[i, c] dG[t, i] + Wu[i, c] dU[t, i]
             g.A = s->Wg; g.A2 = s->Wu; g.lda_m = 1; g.lda_k = C; g.a_outer = I;
-            g.B = s->dG; g.B2 = s->dU; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap;
-            g.M = C; g.N = (int32_t)N; g.n_from_nk = 1; g.K = I;
+            g.B = s->dG; g.B2 = s->dU; g.ldb_n = I; g.ldb_k = 1; g.b_outer = s->cap_k;
+            g.M = C; g.N = NB; g.n_from_nk = 1; g.K = I;
         } else {
-            g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap;
+            g.A = s->dG; g.A2 = s->dU; g.lda_m = I; g.lda_k = 1; g.a_outer = s->cap_k;
             g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = 1; g.ldb_k = C; g.b_outer = I;
-            g.M = (int32_t)N; g.m_from_nk = 1; g.N = C; g.K = I;
+            g.M = NB; g.m_from_nk = 1; g.N = C; g.K = I;
         }
         if (prenorm) { g.in0 = nullptr; g.out0 = s->dY; g.out_fp32 = 1; }   // gradient w.r.t. the normalised rows
         else { g.in0 = s->dOk; g.out0 = dx; }

@@ -15,7 +15,7 @@ enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_ROLE_BASE = 16, ST_WORDS 
 
 // Wait sites reported through the status word when a bounded wait gives up.
 enum : int { SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_TMEM_EMPTY = 3,
-             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6, SITE_EPI_EXCHANGE = 7 };
+             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6, SITE_EPI_EXCHANGE = 7, SITE_KEPT_OVERFLOW = 8 };
 
 // Split-K hand-over between CTAs of one tensor-core GEMM launch: a CTA that computes only part
 // of a tile's K range leaves its fp32 accumulator in its own slot of the workspace and raises one
@@ -150,7 +150,7 @@ enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_
 
 // compact.cu
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
-                           int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s);
+                           int32_t *pos, int32_t *status, int64_t cap, int64_t max_kept, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs &a, cudaStream_t s);
 // kvcache.cu
 cudaError_t launch_kv_compact(const void *src, void *dst, const int32_t *idx, const int32_t *status,

@@ -9,6 +9,9 @@ namespace skipffn {
 //             (inside idx's capacity) are 0, a valid row, so that padded gathers stay in bounds
 //   pos[t]  : rank of token t among kept tokens, or -1 if skipped
 //   status[ST_NK] = Nk
+// If the mask keeps more than `max_kept` tokens (the bound the compacted arrays were sized for), the
+// first max_kept of them are kept, the others are treated as skipped, Nk = max_kept, and the status
+// word reports SKIPFFN_EWORKSPACE: memory stays safe, the results are not those of the mask.
 //
 // k_compact: one CTA per block of 4096 tokens, no communication between CTAs.  A CTA first counts
 // the kept tokens in front of its block by reading that part of the mask itself (at most N bytes,
@@ -38,7 +41,7 @@ __device__ __forceinline__ int block_sum(int v, int *warp_tot)
 
 __global__ void __launch_bounds__(CB_THREADS)
 k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
-          int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
+          int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap, int max_kept)
 {
     __shared__ int warp_tot[CB_THREADS / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -89,11 +92,16 @@ k_compact(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__res
 #pragma unroll
     for (int j = 0; j < CB_PER_THREAD; ++j) {
         if (t0 + j < N) {
-            if ((keep >> j) & 1u) { idx[r] = (int32_t)(t0 + j); pos[t0 + j] = r; ++r; }
+            if (((keep >> j) & 1u) && r < max_kept) { idx[r] = (int32_t)(t0 + j); pos[t0 + j] = r; }
             else pos[t0 + j] = -1;
+            r += (keep >> j) & 1u;
         }
     }
     if (blockIdx.x == gridDim.x - 1) {   // the last block knows the total
+        if (total > max_kept) {
+            total = max_kept;
+            if (tid == 0 && atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_EWORKSPACE) == 0) status[ST_SITE] = SITE_KEPT_OVERFLOW;
+        }
         if (tid == 0) status[ST_NK] = total;
         int64_t end = ((int64_t)total + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
         if (end > cap) end = cap;
@@ -110,7 +118,7 @@ constexpr int CP_J = 16;
 
 __global__ void __launch_bounds__(CP_THREADS)
 k_compact_serial(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t *__restrict__ idx,
-                 int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap)
+                 int32_t *__restrict__ pos, int32_t *__restrict__ status, int64_t cap, int max_kept)
 {
     __shared__ int seg[CP_J * 32];
     __shared__ int slab_total;
@@ -150,8 +158,8 @@ k_compact_serial(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t
             if (t < N) {
                 if ((bal[j] >> lane) & 1u) {
                     int r = carry + seg[j * 32 + warp] + __popc(bal[j] & lt);
-                    idx[r] = (int32_t)t;
-                    pos[t] = r;
+                    if (r < max_kept) { idx[r] = (int32_t)t; pos[t] = r; }
+                    else pos[t] = -1;
                 } else {
                     pos[t] = -1;
                 }
@@ -160,6 +168,10 @@ k_compact_serial(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t
         carry += slab_total;
         __syncthreads();
     }
+    if (carry > max_kept) {
+        carry = max_kept;
+        if (tid == 0 && atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_EWORKSPACE) == 0) status[ST_SITE] = SITE_KEPT_OVERFLOW;
+    }
     if (tid == 0) status[ST_NK] = carry;
     int64_t end = ((int64_t)carry + ROW_PAD - 1) / ROW_PAD * ROW_PAD;
     if (end > cap) end = cap;
@@ -167,12 +179,13 @@ k_compact_serial(const uint8_t *__restrict__ mask, int64_t N, int dense, int32_t
 }
 
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
-                           int32_t *pos, int32_t *status, int64_t cap, cudaStream_t s)
+                           int32_t *pos, int32_t *status, int64_t cap, int64_t max_kept, cudaStream_t s)
 {
+    const int mk = (int)(max_kept < N ? max_kept : N);
     if (N > CB_MAX_N)
-        return launch_pdl(k_compact_serial, dim3(1), dim3(CP_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
+        return launch_pdl(k_compact_serial, dim3(1), dim3(CP_THREADS), s, mask, N, (int)dense, idx, pos, status, cap, mk);
     const unsigned blocks = (unsigned)((N + CB_TOKENS - 1) / CB_TOKENS);
-    return launch_pdl(k_compact, dim3(blocks), dim3(CB_THREADS), s, mask, N, (int)dense, idx, pos, status, cap);
+    return launch_pdl(k_compact, dim3(blocks), dim3(CB_THREADS), s, mask, N, (int)dense, idx, pos, status, cap, mk);
 }
 
 // Row routing.  Unit u < N is token u: a kept token's row goes to dst_compact[pos[u]], a skipped

@@ -61,7 +61,7 @@ extern "C" skipffn_status skipffn_compact_static(const uint8_t *skip_mask, int64
     if (scratch_address(&scratch) != cudaSuccess) return SKIPFFN_ECUDA;
     int32_t *status = scratch, *pos = scratch + ST_WORDS;
     // cap = N: the kernel's padding entries past the kept count stay inside idx[0 .. N-1]
-    if (launch_compact(skip_mask, N, 0, idx, pos, status, N, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    if (launch_compact(skip_mask, N, 0, idx, pos, status, N, N, st) != cudaSuccess) return SKIPFFN_ECUDA;
     if (cudaMemcpyAsync(nk, status + ST_NK, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return SKIPFFN_ECUDA;
     return SKIPFFN_OK;

@@ -222,8 +222,8 @@ static cudaError_t merge_t(const T *X, int64_t n, int C, int k, int dtype, int32
     // 2. the k most distinctive tokens, and the others, each as an ascending index list
     k_rank_select<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(m.avg, n, k, m.drop, m.drop_inv);
     if ((e = cudaMemsetAsync(m.status_k, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, s)) != cudaSuccess) return e;
-    if ((e = launch_compact(m.drop, n, 0, m.kept, m.pos, m.status_k, round_up(n, ROW_PAD) + ROW_PAD, s)) != cudaSuccess) return e;
-    if ((e = launch_compact(m.drop_inv, n, 0, m.rest, m.pos, m.status_r, round_up(n, ROW_PAD) + ROW_PAD, s)) != cudaSuccess) return e;
+    if ((e = launch_compact(m.drop, n, 0, m.kept, m.pos, m.status_k, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
+    if ((e = launch_compact(m.drop_inv, n, 0, m.rest, m.pos, m.status_r, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
     if ((e = cudaMemcpyAsync(kept_out, m.kept, (size_t)k * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess) return e;
     // 3. assignment: unit rows, similarity GEMM, arg max
     if (n_rest > 0) {

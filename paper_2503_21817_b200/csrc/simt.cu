@@ -88,8 +88,8 @@ __global__ void __launch_bounds__(ST_THREADS) k_simt_gemm(GemmArgs a)
             int64_t o = (int64_t)m * a.ldo + n;
             if (EPI == EPI_GATEUP) {             // G, U, H = silu(G) * U   (compacted rows)
                 float u = acc2[DUAL ? i : 0][j];
-                ((T *)a.out0)[o] = from_f32<T>(v);
-                ((T *)a.out1)[o] = from_f32<T>(u);
+                if (a.out0) ((T *)a.out0)[o] = from_f32<T>(v);   // a recomputing forward stores H only
+                if (a.out1) ((T *)a.out1)[o] = from_f32<T>(u);
                 ((T *)a.out2)[o] = from_f32<T>(swiglu(v, u));   // from the fp32 accumulators
             } else if (EPI == EPI_DX && a.out_fp32) {        // pre-norm variant: raw fp32 rows, compact
                 ((float *)a.out0)[o] = v;
@@ -120,8 +120,8 @@ __global__ void __launch_bounds__(ST_THREADS) k_simt_gemm(GemmArgs a)
         for (int m = M + ty; m < end; m += 16)
             for (int n = n0 + tx; n < n0 + ST_BN && n < N; n += 16) {
                 int64_t o = (int64_t)m * a.ldo + n;
-                ((T *)a.out0)[o] = from_f32<T>(0.0f);
-                ((T *)a.out1)[o] = from_f32<T>(0.0f);
+                if (a.out0) ((T *)a.out0)[o] = from_f32<T>(0.0f);
+                if (a.out1) ((T *)a.out1)[o] = from_f32<T>(0.0f);
                 if (EPI == EPI_GATEUP) ((T *)a.out2)[o] = from_f32<T>(0.0f);
             }
     }

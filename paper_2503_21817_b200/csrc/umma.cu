@@ -661,8 +661,14 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
     // token problems: the column extent is the kept count rounded up to the MMA's N granularity;
     // columns nk .. n_tot-1 exist only as padding (their operand rows are zero)
     const int n_tot = TOK ? (p.n_from_nk ? ((nk + 15) & ~15) : p.N) : 0;
-    // accumulator columns per tile (256 unless overridden)
-    const int tile_w = p.force_bn > 0 ? p.force_bn : BN;
+    // accumulator columns per tile: 256 unless overridden; token problems cut the token range into
+    // the same number of tiles but of equal width (320 tokens: 160 + 160 instead of 256 + 64), which
+    // balances the workers and avoids a sliver whose operand loads would cost as much as a full tile's
+    int tile_w = p.force_bn > 0 ? p.force_bn : BN;
+    if (TOK && p.force_bn <= 0 && n_tot > 0) {
+        const int n_tiles = (n_tot + BN - 1) / BN;
+        tile_w = ((n_tot / 16 + n_tiles - 1) / n_tiles) * 16;
+    }
     // tiles of problem g: ids [g_first[g], g_first[g+1]); token problems run the column (token)
     // tile index fastest, so that tiles sharing a weight panel run at the same time
     const int groups = TOK ? 1 : p.groups;
@@ -1437,7 +1443,7 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_wait_skew = g.sk_wait_skew;
     p.a_one = a_one; p.b_one = b_one; p.gu_one = gu_one;
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
-    static const int sk_threshold[6] = {/*GATEUP*/ 64, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 32, /*DX*/ 40, /*PLAIN*/ 32};
+    static const int sk_threshold[6] = {/*GATEUP*/ 16, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 64, /*DX*/ 40, /*PLAIN*/ 32};
     p.streamk = (g.sk_slots && g.sk_flags) ? (g.tune_streamk >= 0 ? g.tune_streamk : sk_threshold[epi]) : 0;
 
     const int tile_w = p.force_bn > 0 ? p.force_bn : BN;   // accumulator columns per tile

@@ -37,14 +37,14 @@ class DeviceWorkload:
 
 
 def run(w, dense=False, path=0, grad_fp32=False, accumulate_dw=False, inplace=False, dev=None,
-        dw_init=None, tune=None):
+        dw_init=None, tune=None, recompute=False, max_kept=None):
     """Forward + backward through the C ABI; returns a dict of device tensors and the context."""
     import torch
     import paper_2503_21817_b200 as sk
     dev = dev or DeviceWorkload(w)
     dt = sk.BF16 if w.dtype == "bf16" else sk.FP32
     ctx = sk.SkipFFN(w.C, w.I, max(w.N, 1), dtype=dt, dense=dense, path=path, grad_fp32=grad_fp32,
-                     accumulate_dw=accumulate_dw)
+                     accumulate_dw=accumulate_dw, recompute=recompute, max_kept=max_kept)
     if tune:
         ctx.tune(**tune)
     x = dev.x.clone()
