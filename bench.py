@@ -719,6 +719,54 @@ def run_merge(args):
                                        "sample": f"first {ns} tokens, keep 32, {dt:.2f} s"}}), flush=True)
 
 
+# ------------------------------------------------------------------------------ role cycle counters
+def run_role_cycles(args):
+    """Where the tensor-core GEMM kernels spend their cycles, per role: needs the instrumented
+    library (python -m paper_2503_21817_b200.build --role-cycles).  For each GEMM launch of one
+    step, averaged over the SM pairs: the MMA issuer's cycles waiting for operand stages and for a
+    free accumulator and its total, the TMA producer's cycles waiting for a free stage, and one
+    epilogue warp's cycles waiting for a finished accumulator and busy."""
+    import paper_2503_21817_b200.binding as binding
+    from paper_2503_21817_b200.build import LIB_ROLE_CYCLES
+    if not os.path.exists(LIB_ROLE_CYCLES):
+        raise SystemExit("build the instrumented library first: python -m paper_2503_21817_b200.build --role-cycles")
+    binding._LIB_PATH = LIB_ROLE_CYCLES
+    import torch
+    import paper_2503_21817_b200 as sk
+    torch.cuda.set_device(0)
+    w = make_workload(args, 0)
+    x, dout, Wg, Wu, Wd = (_h_bf16(a).cuda() for a in (w.x, w.dout, w.W_gate, w.W_up, w.W_down))
+    mask = torch.from_numpy(w.skip_mask).cuda()
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    if args.tune:
+        ctx.tune(**{k: int(v) for k, v in (kv.split("=") for kv in args.tune.split(","))})
+    out, dx = torch.empty_like(x), torch.empty_like(x)
+    dW = [torch.empty_like(t) for t in (Wg, Wu, Wd)]
+
+    def step():
+        ctx.forward(x, mask, Wg, Wu, Wd, out=out)
+        ctx.backward(dout, dx=dx, dW_gate=dW[0], dW_up=dW[1], dW_down=dW[2])
+    for _ in range(max(args.warmup, 3)):
+        step()
+    ctx.poll()
+    status = ctx._view(ctx._ws_ptr, 64, torch.int32)     # the handle's status block; counters from word 16
+    status[16:64] = 0
+    torch.cuda.synchronize()
+    for _ in range(args.steps):
+        step()
+    ctx.poll()
+    v = status.cpu().numpy().astype(np.float64)
+    res = {}
+    for e, name in enumerate(["gateup", "down", "dh", "dw", "dx"]):
+        c = v[16 + 8 * e: 24 + 8 * e]
+        k = max(c[7], 1.0)
+        res[name] = {"issuer_wait_operands": 16 * c[0] / k, "issuer_wait_accumulator": 16 * c[1] / k,
+                     "issuer_total": 16 * c[2] / k, "producer_wait_free_stage": 16 * c[3] / k,
+                     "epilogue_warp_wait": 16 * c[4] / k, "epilogue_warp_busy": 16 * c[5] / k}
+    print(json.dumps({"role_cycles": "SM cycles per SM pair per launch, mean over %d steps" % args.steps,
+                      "config": workload_config(args, w), "kernels": res}), flush=True)
+
+
 # ------------------------------------------------------------------------------ library yardstick
 def run_yardstick(args):
     """Not part of the metric: times the vendor library's plain GEMMs (torch.matmul) on the five
@@ -779,13 +827,17 @@ def main():
                     help="run warmup+steps steps and exit (launch sequence for an ncu capture)")
     ap.add_argument("--sweep", action="store_true",
                     help="skip-ratio sweep at both shapes against the dense comparator (1 GPU)")
+    ap.add_argument("--role-cycles", action="store_true",
+                    help="per-role cycle counters of the GEMM kernels (needs the instrumented library build)")
     ap.add_argument("--yardstick", action="store_true",
                     help="time the vendor library's plain GEMMs on the path's shapes (context only)")
     ap.add_argument("--kv", action="store_true", help="skip KV-cache compaction (Eq. 7) at the 8B cache shape")
     ap.add_argument("--summary", action="store_true", help="adaptive summary token (Eq. 6), forward + backward")
     ap.add_argument("--merge", action="store_true", help="token merge of section 4.1 on one high-resolution sample")
     args = ap.parse_args()
-    if args.merge:
+    if args.role_cycles:
+        run_role_cycles(args)
+    elif args.merge:
         run_merge(args)
     elif args.summary:
         run_summary(args)

@@ -40,7 +40,8 @@ typedef enum {
     SKIPFFN_EWORKSPACE = 3,   /* workspace too small for max_tokens / max_kept; reported by skipffn_poll
                                  when a mask kept more than max_kept tokens */
     SKIPFFN_ECUDA = 4,        /* a CUDA runtime / driver call failed */
-    SKIPFFN_ETIMEOUT = 5      /* a device-side wait hit its limit (reported by skipffn_poll) */
+    SKIPFFN_ETIMEOUT = 5,     /* a device-side wait hit its limit (reported by skipffn_poll) */
+    SKIPFFN_EDEBUG = 6        /* debug handles: a device-side consistency check failed (skipffn_poll) */
 } skipffn_status;
 
 typedef enum { SKIPFFN_BF16 = 0, SKIPFFN_FP32 = 1 } skipffn_dtype;
@@ -114,12 +115,15 @@ void skipffn_saved_destroy(skipffn_saved *saved);
  *   ONE_BOX         1 (default): an operand tile that consists of two 64-wide pieces (the two slabs
  *                   of a transposed operand; the gate and the up rows) is fetched with one 3-D
  *                   TMA box where the arrays allow it; 0: always one 2-D box per piece
+ *   TMA_STORES      1 (default): weight-gradient tiles that overwrite their destination are written
+ *                   with TMA tile stores from shared memory; 0: with per-lane 16-byte stores
  *   LOSE_HANDOVER   debug handles only (EINVAL otherwise): nonzero makes the finishing units of a
  *                   K-split launch wait for a hand-over that never comes, so that the bounded wait
  *                   runs out and skipffn_poll reports SKIPFFN_ETIMEOUT -- the failure path can be
  *                   exercised without any fault */
 typedef enum { SKIPFFN_TUNE_TILE_N = 0, SKIPFFN_TUNE_STREAMK = 1, SKIPFFN_TUNE_STAGES = 2,
-               SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_COUNT = 5 } skipffn_tunable;
+               SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_TMA_STORES = 5,
+               SKIPFFN_TUNE_COUNT = 6 } skipffn_tunable;
 skipffn_status skipffn_tune(skipffn_saved *saved, int32_t what, int32_t value);
 
 /* Mask compaction alone (the retained / skipped split is the same for every decoder layer, so a
@@ -239,8 +243,14 @@ skipffn_status skipffn_get_intermediate(const skipffn_saved *saved, int32_t whic
                                         const void **ptr_dev);
 
 /* Synchronises `stream`, then reads the device status word: returns SKIPFFN_ETIMEOUT (and the
- * site code in *site_out, may be NULL) if a kernel gave up on a wait, SKIPFFN_ECUDA if the
- * stream reports an error, else SKIPFFN_OK.  The word is cleared. */
+ * site code in *site_out, may be NULL) if a kernel gave up on a wait, SKIPFFN_EWORKSPACE if a mask
+ * kept more than max_kept tokens, SKIPFFN_ECUDA if the stream reports an error, else SKIPFFN_OK.
+ * The word is cleared.
+ * Debug handles (cfg.debug = 1) add two checks, both reported as SKIPFFN_EDEBUG: after every mask
+ * compaction the kept-row list is verified on the device (in range, strictly ascending, inverse map
+ * consistent; site 16), and every slab of the workspace is followed by a 1 KiB guard band whose
+ * contents skipffn_poll verifies (site 32 + slab number): a kernel that wrote past its slab shows up
+ * here instead of corrupting a neighbour silently.  Debug handles need slightly more workspace. */
 skipffn_status skipffn_poll(skipffn_saved *saved, void *stream, int32_t *site_out);
 
 /* Per-launch timing for benchmarks.  While enabled, forward / backward record a CUDA event on the

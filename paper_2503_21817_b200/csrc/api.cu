@@ -26,6 +26,7 @@ struct skipffn_saved {
     const void *Wg, *Wu, *Wd;
     int launches[2];
     int32_t sk_epoch;      // flag value of the latest tensor-core GEMM launch (never 0)
+    GuardList guards;      // debug handles: addresses of the guard bands
     int32_t tune[SKIPFFN_TUNE_COUNT];   // skipffn_tune values
     TmapCache tmaps;       // encoded tensor maps of the arrays this handle launches on
     // optional per-launch timing (CUDA events on the caller's stream)
@@ -44,6 +45,9 @@ struct Layout {
     size_t status, idx, pos, Xk, Xn, rstd, saved_total;                  // saved region
     size_t sk_slots, dOk, dG, dU, dY, dg_part, scratch_total;              // scratch region
     size_t G, U, H;                                                        // in saved, or in scratch when recomputing
+    int n_guards;                                                          // debug handles: guard bands behind the slabs
+    size_t guard_off[MAX_GUARDS];
+    bool guard_in_scratch[MAX_GUARDS];
 };
 
 bool valid_cfg(const skipffn_config *c)
@@ -61,7 +65,18 @@ Layout make_layout(const skipffn_config *c, int64_t max_tokens, int64_t max_kept
     const int64_t cap_k = round_up(max_kept > 0 ? max_kept : 1, ROW_PAD);
     const size_t es = c->dtype == SKIPFFN_BF16 ? 2 : 4;
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 1024); return o; };
+    bool in_scratch = false;
+    l.n_guards = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = (size_t)round_up((int64_t)(off + bytes), 1024);
+        if (c->debug && bytes > 0 && l.n_guards < MAX_GUARDS) {   // guard band right behind the slab
+            l.guard_off[l.n_guards] = off;
+            l.guard_in_scratch[l.n_guards++] = in_scratch;
+            off += GUARD_BYTES;
+        }
+        return o;
+    };
     l.status = take((ST_WORDS + SK_FLAG_WORDS) * 4);   // status block, then the hand-over flags
     l.idx = take((size_t)cap * 4);
     l.pos = take((size_t)cap * 4);
@@ -75,6 +90,7 @@ Layout make_layout(const skipffn_config *c, int64_t max_tokens, int64_t max_kept
     }
     l.saved_total = off;
     off = 0;
+    in_scratch = true;
     l.sk_slots = take(c->dtype == SKIPFFN_BF16 ? (size_t)SK_MAX_CTAS * SK_SLOT_BYTES : 0);
     l.dOk = take((size_t)cap_k * c->C * es);
     l.dG = take((size_t)cap_k * c->I * es);
@@ -142,8 +158,19 @@ GemmArgs base_args(skipffn_saved *s)
     // flag value that nothing writes, so their bounded wait runs out
     g.sk_wait_skew = (s->cfg.debug && s->tune[SKIPFFN_TUNE_LOSE_HANDOVER]) ? 0x40000000 : 0;
     g.one_box_loads = s->tune[SKIPFFN_TUNE_ONE_BOX];
+    g.tma_stores = s->tune[SKIPFFN_TUNE_TMA_STORES];
     g.tmaps = &s->tmaps;
     return g;
+}
+
+// first use of a handle: clear the status block and the hand-over flags; debug handles fill their guard bands
+cudaError_t first_use(skipffn_saved *s, cudaStream_t st)
+{
+    if (s->planned_N >= 0) return cudaSuccess;
+    cudaError_t e = cudaMemsetAsync(s->status, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, st);
+    for (int i = 0; e == cudaSuccess && i < s->guards.n; ++i)
+        e = cudaMemsetAsync(const_cast<void *>(s->guards.ptr[i]), GUARD_BYTE, GUARD_BYTES, st);
+    return e;
 }
 
 skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int which, cudaStream_t st)
@@ -154,6 +181,7 @@ skipffn_status do_plan(skipffn_saved *s, const uint8_t *mask, int64_t N, int whi
                 return launch_compact(mask, N, s->cfg.dense, s->idx, s->pos, s->status, s->cap, s->max_kept, st);
             }) != cudaSuccess)
             return SKIPFFN_ECUDA;
+        if (s->cfg.debug && launch_check_kept(s->idx, s->pos, s->status, N, st) != cudaSuccess) return SKIPFFN_ECUDA;
     } else if (cudaMemsetAsync(s->status, 0, 4, st) != cudaSuccess) {
         return SKIPFFN_ECUDA;
     }
@@ -228,6 +256,9 @@ skipffn_status skipffn_saved_create_split(skipffn_saved **saved, const skipffn_c
     s->planned_N = -1;
     s->tune[SKIPFFN_TUNE_STREAMK] = -1;
     s->tune[SKIPFFN_TUNE_ONE_BOX] = 1;
+    s->tune[SKIPFFN_TUNE_TMA_STORES] = 1;
+    s->guards.n = l.n_guards;
+    for (int i = 0; i < l.n_guards; ++i) s->guards.ptr[i] = (l.guard_in_scratch[i] ? x : w) + l.guard_off[i];
     *saved = s;
     return SKIPFFN_OK;
 }
@@ -303,8 +334,7 @@ skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t 
     if (!skip_mask && !s->cfg.dense && N > 0) return SKIPFFN_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     // the status word is cleared together with the first plan of a handle
-    if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, st) != cudaSuccess)
-        return SKIPFFN_ECUDA;
+    if (first_use(s, st) != cudaSuccess) return SKIPFFN_ECUDA;
     s->launches[0] = 0;
     s->forwarded = 0;
     return do_plan(s, skip_mask, N, 0, st);
@@ -354,8 +384,7 @@ static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_
     const int C = s->cfg.C, I = s->cfg.I;
     s->forwarded = 0;
     if (skip_mask || s->cfg.dense || N == 0) {
-        if (s->planned_N < 0 && cudaMemsetAsync(s->status, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, st) != cudaSuccess)
-            return SKIPFFN_ECUDA;
+        if (first_use(s, st) != cudaSuccess) return SKIPFFN_ECUDA;
         s->launches[0] = 0;
         skipffn_status r = do_plan(s, skip_mask, N, 0, st);
         if (r != SKIPFFN_OK) return r;
@@ -640,6 +669,7 @@ skipffn_status skipffn_poll(skipffn_saved *s, void *stream, int32_t *site_out)
 {
     if (!s) return SKIPFFN_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
+    if (s->cfg.debug && s->planned_N >= 0 && launch_check_guards(s->guards, s->status, st) != cudaSuccess) return SKIPFFN_ECUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return SKIPFFN_ECUDA;
     int32_t w[3] = {0, 0, 0};
     if (cudaMemcpy(w, s->status, sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess) return SKIPFFN_ECUDA;
@@ -685,6 +715,7 @@ const char *skipffn_strerror(skipffn_status st)
     case SKIPFFN_EWORKSPACE: return "workspace too small";
     case SKIPFFN_ECUDA: return "CUDA call failed";
     case SKIPFFN_ETIMEOUT: return "device-side wait timed out";
+    case SKIPFFN_EDEBUG: return "debug check failed";
     }
     return "unknown status";
 }

@@ -15,7 +15,8 @@ enum : int { ST_NK = 0, ST_STATUS = 1, ST_SITE = 2, ST_ROLE_BASE = 16, ST_WORDS 
 
 // Wait sites reported through the status word when a bounded wait gives up.
 enum : int { SITE_PRODUCER_EMPTY = 1, SITE_MMA_FULL = 2, SITE_MMA_TMEM_EMPTY = 3,
-             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6, SITE_EPI_EXCHANGE = 7, SITE_KEPT_OVERFLOW = 8 };
+             SITE_EPI_TMEM_FULL = 4, SITE_TEARDOWN = 5, SITE_EPI_PARTIAL = 6, SITE_EPI_EXCHANGE = 7, SITE_KEPT_OVERFLOW = 8,
+             SITE_DEBUG_KEPT_LIST = 16, SITE_DEBUG_GUARD_BASE = 32 /* + index of the slab whose guard band changed */ };
 
 // Split-K hand-over between CTAs of one tensor-core GEMM launch: a CTA that computes only part
 // of a tile's K range leaves its fp32 accumulator in its own slot of the workspace and raises one
@@ -141,6 +142,7 @@ struct GemmArgs {
     // tensor-core path: tuning overrides of the handle (0 / -1 = defaults) and its tensor-map cache
     int32_t tune_tile_n, tune_stages, tune_streamk;
     int32_t one_box_loads;      // 1: load an operand tile with one 3-D box where the arrays allow it
+    int32_t tma_stores;         // 1: weight-gradient tiles leave through TMA tile stores (overwrite mode)
     TmapCache *tmaps;
 };
 
@@ -152,6 +154,11 @@ enum Epilogue : int { EPI_GATEUP = 0, EPI_DOWN = 1, EPI_DH = 2, EPI_DW = 3, EPI_
 cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_t *idx,
                            int32_t *pos, int32_t *status, int64_t cap, int64_t max_kept, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs &a, cudaStream_t s);
+// debug handles: guard bands behind the workspace slabs, and the invariants of the kept-row list
+constexpr int GUARD_BYTES = 1024, GUARD_BYTE = 0xA5, MAX_GUARDS = 24;
+struct GuardList { int n; const void *ptr[MAX_GUARDS]; };
+cudaError_t launch_check_kept(const int32_t *idx, const int32_t *pos, int32_t *status, int64_t N, cudaStream_t s);
+cudaError_t launch_check_guards(const GuardList &g, int32_t *status, cudaStream_t s);
 // kvcache.cu
 cudaError_t launch_kv_compact(const void *src, void *dst, const int32_t *idx, const int32_t *status,
                               int64_t planes, int64_t N, int64_t dst_rows, int64_t row_bytes,

@@ -188,6 +188,44 @@ cudaError_t launch_compact(const uint8_t *mask, int64_t N, int32_t dense, int32_
     return launch_pdl(k_compact, dim3(blocks), dim3(CB_THREADS), s, mask, N, (int)dense, idx, pos, status, cap, mk);
 }
 
+// Debug handles: check the kept-row list against its own invariants (in range, strictly ascending,
+// consistent with the inverse map) and report a violation through the status word.
+__global__ void k_check_kept(const int32_t *__restrict__ idx, const int32_t *__restrict__ pos,
+                             int32_t *__restrict__ status, int64_t N)
+{
+    const int nk = status[ST_NK];
+    bool bad = nk < 0 || nk > N;
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; !bad && r < nk; r += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t t = idx[r];
+        bad = t < 0 || t >= N || (r > 0 && idx[r - 1] >= t) || pos[t] != (int32_t)r;
+    }
+    if (bad && atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_EDEBUG) == 0) status[ST_SITE] = SITE_DEBUG_KEPT_LIST;
+}
+
+// Debug handles: every slab of the workspace is followed by a guard band filled with GUARD_BYTE; a
+// kernel that wrote past the end of its slab leaves a different byte there.
+__global__ void k_check_guards(GuardList g, int32_t *__restrict__ status)
+{
+    const uint32_t want = 0x01010101u * GUARD_BYTE;
+    const uint32_t *p = reinterpret_cast<const uint32_t *>(g.ptr[blockIdx.x]);
+    bool bad = false;
+    for (int i = threadIdx.x; i < GUARD_BYTES / 4; i += blockDim.x) bad |= p[i] != want;
+    if (bad && atomicCAS(&status[ST_STATUS], 0, (int)SKIPFFN_EDEBUG) == 0) status[ST_SITE] = SITE_DEBUG_GUARD_BASE + (int)blockIdx.x;
+}
+
+cudaError_t launch_check_kept(const int32_t *idx, const int32_t *pos, int32_t *status, int64_t N, cudaStream_t s)
+{
+    k_check_kept<<<64, 256, 0, s>>>(idx, pos, status, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_check_guards(const GuardList &g, int32_t *status, cudaStream_t s)
+{
+    if (g.n <= 0) return cudaSuccess;
+    k_check_guards<<<g.n, 128, 0, s>>>(g, status);
+    return cudaGetLastError();
+}
+
 // Row routing.  Unit u < N is token u: a kept token's row goes to dst_compact[pos[u]], a skipped
 // token's row goes to dst_identity[u] (byte copy; omitted when dst_identity is null or the
 // source itself).  Units u >= N zero the padding rows Nk .. round_up(Nk, ROW_PAD)-1 of

@@ -192,6 +192,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
 }
+// Tile store shared -> global (clipped at the tensor's edges), tracked in the issuing thread's bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src),
+                 "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// wait until at most N of this thread's bulk groups still READ their shared-memory source
+template <int N> __device__ __forceinline__ void tma_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -302,6 +315,13 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrive without memory ordering.  Handing an accumulator back orders only tensor-memory reads, which
+// the tcgen05 wait / fence before the arrive already does; a releasing arrive would in addition wait
+// until the epilogue's outstanding global stores are visible (measured: about 2400 cycles per tile).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // TMA load into this CTA's shared memory whose bytes are counted on the pair leader's mbarrier
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1,
                                                  uint32_t leader_bar)
@@ -407,6 +427,7 @@ struct UmmaParams {
     // one-instruction operand loads (see TmapSet): which of them the host could encode
     int32_t a_one, b_one;            // MN-major operand: both 64-wide slabs of a CTA's 128 in one 3-D box
     int32_t gu_one;                  // gate/up: gate and up rows in one 3-D box; 2 = the up rows come first
+    int32_t dw_tma;                  // weight gradients (overwrite mode): tiles leave through TMA stores (maps O[g])
 };
 
 // Tensor maps of one launch.  A, B, A2, B2, A3: 2-D maps (box = 64 elements of the contiguous
@@ -414,8 +435,9 @@ struct UmmaParams {
 // whole half of a full-width token tile arrives with one instruction.  A1, A21, A31, B1, B21: 3-D views
 // of MN-major arrays [K rows, 64-wide slab, 64 columns] whose box holds two slabs (128 columns); for
 // gate/up A1 is the 3-D view [K, weight row, {gate, up}] of the two weight matrices.
+// O[g]: the output matrix of weight-gradient problem g, box = 32 rows x 64 bytes, 64-byte swizzle.
 struct alignas(64) TmapSet {
-    CUtensorMap A, B, A2, B2, A3, Bw, B2w, A1, A21, A31, B1, B21;
+    CUtensorMap A, B, A2, B2, A3, Bw, B2w, A1, A21, A31, B1, B21, O[3];
 };
 
 struct alignas(8) SmemCtl {
@@ -880,6 +902,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
         const uint32_t xbuf = epi_bufs + EPI_WARPS * EPI_BUF_BYTES + xpair * X_BUF_BYTES;
         const uint32_t xfull_bar = smem_u32(&ctl->xfull[xpair]), xempty_bar = smem_u32(&ctl->xempty[xpair]);
         uint32_t xcount = 0;            // chunks exchanged so far by this warp
+        uint32_t tbuf = 0;              // weight gradients: staging buffers handed to TMA stores so far
         // accumulators are handed back on the leader's barrier, which its MMA warp waits on
         const uint32_t empty_bar0 = smem_u32(&ctl->tmem_empty[0]);
         // hand-over slots: a warp reads back exactly the words the same warp of the producing CTA wrote
@@ -1126,7 +1149,41 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
                     uint32_t w[16];
                     const int64_t o = (int64_t)m * p.gldo[tl.g] + n;
                     char *row = row_valid ? (char *)p.gout[tl.g] + o * esz : nullptr;
-                    if (p.out_fp32) {
+                    if (p.dw_tma) {
+                        // overwrite mode: the 32-row x 64-byte chunk is staged (same XOR layout as the
+                        // 64-byte TMA swizzle) and leaves as one tile store, which also clips at the
+                        // matrix edges; two staging buffers per warp, so a store still reading one of
+                        // them overlaps the next chunk
+                        const CUtensorMap *mo = tl.g == 2 ? &tm.O[2] : (tl.g == 1 ? &tm.O[1] : &tm.O[0]);
+                        const int m_warp = m - lane;
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            if (!p.out_fp32 && hh == 1) break;
+                            if (p.out_fp32) {
+#pragma unroll
+                                for (int q = 0; q < 16; ++q) w[q] = r[hh * 16 + q];
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 16; ++q) w[q] = pack_bf16(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+                            }
+                            const uint32_t sb2 = (tbuf & 1) ? sbuf + EPI_WARPS * EPI_BUF_BYTES : sbuf;
+                            ++tbuf;
+                            if (lane == 0) tma_store_wait_read<1>();   // the store that last used this buffer has read it
+                            __syncwarp();
+                            const int sw = (lane >> 1) & 3;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sb2 + lane * 64 + ((c ^ sw) << 4)),
+                                             "r"(w[4 * c]), "r"(w[4 * c + 1]), "r"(w[4 * c + 2]), "r"(w[4 * c + 3])
+                                             : "memory");
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            __syncwarp();
+                            if (lane == 0) {
+                                tma_store_2d(mo, sb2, n + hh * 16, m_warp);
+                                tma_store_commit();
+                            }
+                        }
+                    } else if (p.out_fp32) {
 #pragma unroll
                         for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
@@ -1163,12 +1220,13 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
                 __syncwarp();
                 if (lane == 0) {
                     const uint32_t bar = empty_bar0 + acc * 8;
-                    if (PAIR) mbar_arrive_cluster(mapa_rank(bar, 0));
+                    if (PAIR) mbar_arrive_cluster_relaxed(mapa_rank(bar, 0));
                     else mbar_arrive(bar);
                 }
             }
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
+        if (!TOK && lane == 0) tma_store_wait_read<0>();   // the staging buffers are free before the CTA gives them up
 #ifdef SKIPFFN_ROLE_CYCLES
         if (ew == 0 && lane == 0 && rank == 0) {
             atomicAdd(&p.status[ST_ROLE_BASE + 8 * EPI + 4], (int)(role_wait >> 4));
@@ -1247,6 +1305,42 @@ static bool make_map(CUtensorMap *m, TmapCache *cache, const void *base, int64_t
     if (cache) {
         const int i = cache->used < TMAP_CACHE_ENTRIES ? cache->used++ : (cache->next++ % TMAP_CACHE_ENTRIES);
         cache->key[i] = TmapKey{base, inner, outer, pitch, box_outer, dim2, stride2_bytes};
+        memcpy(cache->map[i], m, TMAP_BYTES);
+    }
+    return true;
+}
+
+// Output matrix of a weight-gradient problem for TMA tile stores: row-major [rows, cols] with row
+// pitch `pitch` elements of 2 or 4 bytes; box = 32 rows x 64 bytes, 64-byte swizzle (the layout of the
+// epilogue's staging buffers).
+static bool make_out_map(CUtensorMap *m, TmapCache *cache, const void *base, int64_t rows, int64_t cols, int64_t pitch,
+                         bool fp32)
+{
+    if (!base) return false;
+    const int kind = fp32 ? -2 : -1;   // kept apart from operand maps in the cache
+    if (cache) {
+        for (int i = 0; i < cache->used; ++i) {
+            const TmapKey &k = cache->key[i];
+            if (k.base == base && k.inner == cols && k.outer == rows && k.pitch == pitch && k.box_outer == 32 && k.dim2 == kind) {
+                memcpy(m, cache->map[i], TMAP_BYTES);
+                return true;
+            }
+        }
+    }
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const int esz = fp32 ? 4 : 2;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch * esz};
+    cuuint32_t box[2] = {(cuuint32_t)(64 / esz), 32u};
+    cuuint32_t es[2] = {1u, 1u};
+    CUresult r = enc(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                     const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return false;
+    if (cache) {
+        const int i = cache->used < TMAP_CACHE_ENTRIES ? cache->used++ : (cache->next++ % TMAP_CACHE_ENTRIES);
+        cache->key[i] = TmapKey{base, cols, rows, pitch, 32, kind, 0};
         memcpy(cache->map[i], m, TMAP_BYTES);
     }
     return true;
@@ -1442,6 +1536,14 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_epoch = g.sk_epoch;
     p.sk_wait_skew = g.sk_wait_skew;
     p.a_one = a_one; p.b_one = b_one; p.gu_one = gu_one;
+    // weight gradients that overwrite their destination leave through TMA tile stores
+    p.dw_tma = 0;
+    tm.O[0] = tm.O[1] = tm.O[2] = tm.A;
+    if (!tok && !g.accumulate && g.tma_stores) {
+        p.dw_tma = 1;
+        for (int i = 0; i < n && p.dw_tma; ++i)
+            if (!make_out_map(&tm.O[i], gs[i].tmaps, gs[i].out0, gs[i].M, gs[i].N, gs[i].ldo, gs[i].out_fp32 != 0)) p.dw_tma = 0;
+    }
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
     static const int sk_threshold[6] = {/*GATEUP*/ 16, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 64, /*DX*/ 40, /*PLAIN*/ 32};
     p.streamk = (g.sk_slots && g.sk_flags) ? (g.tune_streamk >= 0 ? g.tune_streamk : sk_threshold[epi]) : 0;

@@ -132,16 +132,19 @@ def test_k_split_schedule_forced_on_and_off(min_saving, case):
     _compare(w, run(w, tune=dict(streamk=min_saving)), _oracle_all(w))
 
 
-@pytest.mark.parametrize("one_box", [0, 1])
-def test_operand_tiles_fetched_with_one_or_two_boxes(one_box):
-    # shapes whose extents are multiples of 64, so that the one-box (3-D) operand loads apply; both
-    # ways of fetching must give the same bits
-    w = wl.small_case(27, "bf16", 512, 1024, 3, 20, 300, 0.5)
-    r = run(w, tune=dict(one_box=one_box))
-    _compare(w, r, _oracle_all(w))
-    ref = run(w, tune=dict(one_box=1 - one_box))
-    for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
-        assert np.array_equal(bits(r[k]), bits(ref[k])), k
+@pytest.mark.parametrize("knob", ["one_box", "tma_stores"])
+@pytest.mark.parametrize("grad_fp32", [False, True])
+def test_alternative_load_and_store_paths_give_the_same_bits(knob, grad_fp32):
+    # operand tiles fetched with one 3-D box or one 2-D box per piece; weight-gradient tiles written
+    # by TMA tile stores or per-lane stores.  Shapes: multiples of 64 (where the one-box loads
+    # apply) and ragged ones (where the tile stores clip at the matrix edges).
+    for w in (wl.small_case(27, "bf16", 512, 1024, 3, 20, 300, 0.5), wl.small_case(28, "bf16", 576, 1000, 3, 20, 200, 0.6)):
+        ref = _oracle_all(w)
+        a = run(w, grad_fp32=grad_fp32, tune={knob: 1})
+        b = run(w, grad_fp32=grad_fp32, tune={knob: 0})
+        _compare(w, a, ref)
+        for k in ("out", "dx", "dW_gate", "dW_up", "dW_down"):
+            assert np.array_equal(bits(a[k]), bits(b[k])), k
 
 
 def test_contiguous_span_layout():
@@ -403,6 +406,39 @@ def test_lost_hand_over_is_reported_and_the_context_stays_usable():
     out = ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
     ctx.poll()                                              # status word was cleared by the failed poll
     check(to_host(out), oracle.forward(w.x, w.skip_mask, w.W_gate, w.W_up, w.W_down), "bf16", "out after recovery")
+
+
+def test_debug_handle_checks_kept_list_and_guard_bands():
+    # A debug handle verifies the kept-row list on the device after every compaction and keeps a
+    # guard band behind every workspace slab, which skipffn_poll checks.  A normal run raises
+    # nothing and gives the same bits as a plain handle; a byte changed inside a guard band (done
+    # here from the host, as an overrunning kernel would) is reported as SKIPFFN_EDEBUG.
+    import torch
+    sk = _sk()
+    w = wl.small_case(29, "bf16", 256, 512, 2, 16, 120, 0.7)
+    dev = DeviceWorkload(w)
+    plain = sk.SkipFFN(w.C, w.I, w.N)
+    ctx = sk.SkipFFN(w.C, w.I, w.N, debug=True)
+    assert ctx.saved_bytes > plain.saved_bytes
+    out = ctx.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
+    res = ctx.backward(dev.dout)
+    ctx.poll()
+    ref_out = plain.forward(dev.x, dev.mask, dev.W_gate, dev.W_up, dev.W_down)
+    ref = plain.backward(dev.dout)
+    plain.poll()
+    for a, b in zip((out,) + tuple(res), (ref_out,) + tuple(ref)):
+        assert np.array_equal(bits(a), bits(b))
+    # find a guard band (1 KiB of the fill byte) in the saved region and damage it
+    ws = ctx.workspace
+    is_fill = (ws == 0xA5).to(torch.int32)
+    runs = torch.nn.functional.avg_pool1d(is_fill.float()[None, None], 1024, stride=1)[0, 0]
+    start = int(torch.nonzero(runs == 1.0)[0, 0])
+    ws[start + 100] = 0
+    with pytest.raises(sk.SkipFFNError) as e:
+        ctx.poll()
+    assert e.value.status == 6
+    ws[start + 100] = 0xA5
+    ctx.poll()                                                        # repaired: clean again
 
 
 def test_single_cta_launch_shape_in_a_fresh_process():
