@@ -117,13 +117,17 @@ void skipffn_saved_destroy(skipffn_saved *saved);
  *                   TMA box where the arrays allow it; 0: always one 2-D box per piece
  *   TMA_STORES      1 (default): weight-gradient tiles that overwrite their destination are written
  *                   with TMA tile stores from shared memory; 0: with per-lane 16-byte stores
+ *   GATHER          1: the gate/up and dH GEMMs fetch their token rows straight from x / dout with
+ *                   tile::gather4 TMA loads driven by the kept-row list, instead of from the
+ *                   compacted copy (which is still made: the weight gradients and the residual
+ *                   read it).  0 (default): compacted copy, which measured faster
  *   LOSE_HANDOVER   debug handles only (EINVAL otherwise): nonzero makes the finishing units of a
  *                   K-split launch wait for a hand-over that never comes, so that the bounded wait
  *                   runs out and skipffn_poll reports SKIPFFN_ETIMEOUT -- the failure path can be
  *                   exercised without any fault */
 typedef enum { SKIPFFN_TUNE_TILE_N = 0, SKIPFFN_TUNE_STREAMK = 1, SKIPFFN_TUNE_STAGES = 2,
-               SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_TMA_STORES = 5,
-               SKIPFFN_TUNE_COUNT = 6 } skipffn_tunable;
+               SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_TMA_STORES = 5, SKIPFFN_TUNE_GATHER = 6,
+               SKIPFFN_TUNE_COUNT = 7 } skipffn_tunable;
 skipffn_status skipffn_tune(skipffn_saved *saved, int32_t what, int32_t value);
 
 /* Mask compaction alone (the retained / skipped split is the same for every decoder layer, so a

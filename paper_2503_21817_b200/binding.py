@@ -24,7 +24,7 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_workspace_bytes_kept", "skipffn_saved_create_kept", "skipffn_saved_create_split"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
-TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4, "tma_stores": 5}
+TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4, "tma_stores": 5, "gather": 6}
 PROFILE_SLOTS = ["compact", "route_x", "gateup", "down", "route_dout", "dh", "dw_down", "dw_gate",
                  "dw_up", "dx", "norm_bwd", "recompute"]
 

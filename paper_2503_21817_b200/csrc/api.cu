@@ -344,7 +344,8 @@ skipffn_status skipffn_plan(skipffn_saved *s, const uint8_t *skip_mask, int64_t 
 // variant).  The tensor-core kernels take the weights as the A operand (weight rows along the
 // accumulator rows) and the token rows as B; the plain-FMA kernels the other way round.
 // `store_gu` = 0 writes H only.
-static cudaError_t gate_up(skipffn_saved *s, int slot, int32_t NB, bool store_gu, cudaStream_t st)
+static cudaError_t gate_up(skipffn_saved *s, int slot, int32_t NB, bool store_gu, cudaStream_t st,
+                           const void *gather_x = nullptr, int64_t gather_rows = 0)
 {
     const int C = s->cfg.C, I = s->cfg.I;
     const void *Xrows = s->cfg.prenorm ? s->Xn : s->Xk;
@@ -353,6 +354,7 @@ static cudaError_t gate_up(skipffn_saved *s, int slot, int32_t NB, bool store_gu
         g.A = s->Wg; g.A2 = s->Wu; g.lda_m = C; g.lda_k = 1; g.a_outer = I;
         g.B = Xrows; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap_k;
         g.M = I; g.N = NB; g.n_from_nk = 1; g.K = C;
+        if (s->tune[SKIPFFN_TUNE_GATHER] && !s->cfg.prenorm) { g.gather_src = gather_x; g.gather_rows = gather_rows; }
     } else {
         g.A = Xrows; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap_k;
         g.B = s->Wg; g.B2 = s->Wu; g.ldb_n = C; g.ldb_k = 1; g.b_outer = I;
@@ -407,7 +409,9 @@ static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_
     const int32_t NB = (int32_t)(N < s->max_kept ? N : s->max_kept);   // host bound of the kept count
     const bool tc = use_umma(s);
     // a recomputing handle keeps only H (for the down projection); its backward computes G, U, H again
-    if (gate_up(s, SLOT_GATEUP, NB, !s->cfg.recompute, st) != cudaSuccess) return SKIPFFN_ECUDA;
+    // (the gathering variant reads x itself, so it cannot be used when out aliases x: the down
+    // projection of an earlier tile may already have overwritten rows -- not here, gate/up ends first)
+    if (gate_up(s, SLOT_GATEUP, NB, !s->cfg.recompute, st, x, N) != cudaSuccess) return SKIPFFN_ECUDA;
 
     // out[idx[r]] = Xk[r] + H Wd^T
     GemmArgs g = base_args(s);
@@ -477,6 +481,7 @@ static skipffn_status backward_impl(const void *dout, skipffn_saved *s, void *dx
             g.A = s->Wd; g.lda_m = 1; g.lda_k = I; g.a_outer = C;
             g.B = s->dOk; g.ldb_n = C; g.ldb_k = 1; g.b_outer = s->cap_k;
             g.M = I; g.N = NB; g.n_from_nk = 1; g.K = C;
+            if (s->tune[SKIPFFN_TUNE_GATHER]) { g.gather_src = dout; g.gather_rows = N; }
         } else {
             g.A = s->dOk; g.lda_m = C; g.lda_k = 1; g.a_outer = s->cap_k;
             g.B = s->Wd; g.ldb_n = 1; g.ldb_k = I; g.b_outer = C;

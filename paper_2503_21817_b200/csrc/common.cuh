@@ -143,6 +143,10 @@ struct GemmArgs {
     int32_t tune_tile_n, tune_stages, tune_streamk;
     int32_t one_box_loads;      // 1: load an operand tile with one 3-D box where the arrays allow it
     int32_t tma_stores;         // 1: weight-gradient tiles leave through TMA tile stores (overwrite mode)
+    // gate/up, dH (tensor-core path): non-null = fetch the token operand from this [gather_rows, K]
+    // array through the kept-row list instead of from B (its compacted copy)
+    const void *gather_src;
+    int64_t gather_rows;
     TmapCache *tmaps;
 };
 

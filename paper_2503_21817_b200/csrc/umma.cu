@@ -192,6 +192,25 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
         : "memory");
 }
+// Four rows of a 2-D tensor (row indices r0..r3, 64 elements from column c0) into four consecutive
+// 128-byte rows of shared memory; the tensor map's box is one row high.  A row index outside the
+// tensor reads as zeros.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, int c0, int4 r, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap *map, int c0, int4 r, uint32_t leader_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.cta_group::2 "
+        "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(map), "r"(c0), "r"(r.x), "r"(r.y), "r"(r.z), "r"(r.w), "r"(leader_bar)
+        : "memory");
+}
 // Tile store shared -> global (clipped at the tensor's edges), tracked in the issuing thread's bulk groups
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1)
 {
@@ -428,6 +447,10 @@ struct UmmaParams {
     int32_t a_one, b_one;            // MN-major operand: both 64-wide slabs of a CTA's 128 in one 3-D box
     int32_t gu_one;                  // gate/up: gate and up rows in one 3-D box; 2 = the up rows come first
     int32_t dw_tma;                  // weight gradients (overwrite mode): tiles leave through TMA stores (maps O[g])
+    // gate/up and dH: fetch the token operand straight from the caller's [tokens, C] array with
+    // tile::gather4 loads driven by the kept-row list (map Bg) instead of from the compacted copy
+    int32_t gather;
+    int32_t n_rows;                  // rows of the gathered array (an index >= n_rows reads as zeros)
 };
 
 // Tensor maps of one launch.  A, B, A2, B2, A3: 2-D maps (box = 64 elements of the contiguous
@@ -437,7 +460,7 @@ struct UmmaParams {
 // gate/up A1 is the 3-D view [K, weight row, {gate, up}] of the two weight matrices.
 // O[g]: the output matrix of weight-gradient problem g, box = 32 rows x 64 bytes, 64-byte swizzle.
 struct alignas(64) TmapSet {
-    CUtensorMap A, B, A2, B2, A3, Bw, B2w, A1, A21, A31, B1, B21, O[3];
+    CUtensorMap A, B, A2, B2, A3, Bw, B2w, A1, A21, A31, B1, B21, O[3], Bg;
 };
 
 struct alignas(8) SmemCtl {
@@ -739,7 +762,61 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0 && !zero_acc) {
+        if ((EPI == EPI_GATEUP || EPI == EPI_DH) && p.gather && !zero_acc) {
+            // Gathering variant: the whole warp takes part.  Lane l fetches rows 4l .. 4l+3 of this
+            // CTA's token rows with one gather4 load per K-block; lane 0 also posts the byte count and
+            // loads the weight tile.
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int si = 0; ok && si < num_segs; ++si) {
+                const Seg sg = sched.get(si);
+                const TileLoc tl = locate(sg.tile);
+                const int bn_cta = tl.bn / SPLIT;
+                const int rows4 = (bn_cta + 3) >> 2;                     // gather4 loads of this CTA per K-block
+                const uint32_t stage_tx = SPLIT * (A_BYTES + rows4 * 512);
+                const int m0 = GATEUP ? tl.m0 + (int)rank * (BM / 2) : tl.m0 + (int)rank * BM;
+                const int nb0 = tl.n0 + (int)rank * bn_cta;
+                int4 rows = make_int4(p.n_rows, p.n_rows, p.n_rows, p.n_rows);
+                if (lane < rows4) {
+                    const int r0 = nb0 + 4 * lane;
+                    if (r0 + 0 < nk) rows.x = p.idx[r0 + 0];
+                    if (r0 + 1 < nk) rows.y = p.idx[r0 + 1];
+                    if (r0 + 2 < nk) rows.z = p.idx[r0 + 2];
+                    if (r0 + 3 < nk) rows.w = p.idx[r0 + 3];
+                }
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+                    ok = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1, abort_flag, p.status, SITE_PRODUCER_EMPTY);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const int k0 = kb * BK;
+                    const uint32_t own_bar = smem_u32(&ctl->full[stage]);
+                    const uint32_t bar = PAIR ? mapa_rank(own_bar, 0) : own_bar;
+                    const uint32_t sa = tiles + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    if (lane == 0) {
+                        if (rank == 0) mbar_expect_tx(own_bar, stage_tx);
+                        if (GATEUP) {
+                            if (p.gu_one) {
+                                if (PAIR) tma_load_3d_pair(sa, &tm.A1, k0, m0, 0, bar); else tma_load_3d(sa, &tm.A1, k0, m0, 0, bar);
+                            } else {
+                                if (PAIR) { tma_load_2d_pair(sa, &tmA, k0, m0, bar); tma_load_2d_pair(sa + CHUNK_BYTES, &tmA2, k0, m0, bar); }
+                                else { tma_load_2d(sa, &tmA, k0, m0, bar); tma_load_2d(sa + CHUNK_BYTES, &tmA2, k0, m0, bar); }
+                            }
+                        } else {   // dH: the transposed weight operand in two 64-wide slabs
+#pragma unroll
+                            for (int j = 0; j < BM / 64; ++j) {
+                                if (PAIR) tma_load_2d_pair(sa + j * CHUNK_BYTES, &tmA, m0 + 64 * j, k0, bar);
+                                else tma_load_2d(sa + j * CHUNK_BYTES, &tmA, m0 + 64 * j, k0, bar);
+                            }
+                        }
+                    }
+                    if (lane < rows4) {
+                        if (PAIR) tma_gather4_pair(sb + lane * 512, &tm.Bg, k0, rows, bar);
+                        else tma_gather4(sb + lane * 512, &tm.Bg, k0, rows, bar);
+                    }
+                    if (++stage == nst) { stage = 0; phase ^= 1; }
+                }
+            }
+        } else if (lane == 0 && !zero_acc) {
             prefetch_tmap(&tmA);
             prefetch_tmap(&tmB);
             if (p.segments == 2 || groups > 1) prefetch_tmap(&tmB2);
@@ -1536,6 +1613,13 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     p.sk_epoch = g.sk_epoch;
     p.sk_wait_skew = g.sk_wait_skew;
     p.a_one = a_one; p.b_one = b_one; p.gu_one = gu_one;
+    // gate/up, dH: token rows gathered from the caller's array by the kept-row list (SM-pair shape only)
+    p.gather = 0; p.n_rows = 0;
+    tm.Bg = tm.B;
+    if ((epi == EPI_GATEUP || epi == EPI_DH) && g.gather_src && g.idx &&
+        make_map(&tm.Bg, g.tmaps, g.gather_src, (int64_t)g.K, g.gather_rows, g.ldb_n, 1)) {
+        p.gather = 1; p.n_rows = (int32_t)g.gather_rows;
+    }
     // weight gradients that overwrite their destination leave through TMA tile stores
     p.dw_tma = 0;
     tm.O[0] = tm.O[1] = tm.O[2] = tm.A;
@@ -1545,7 +1629,7 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
             if (!make_out_map(&tm.O[i], gs[i].tmaps, gs[i].out0, gs[i].M, gs[i].N, gs[i].ldo, gs[i].out_fp32 != 0)) p.dw_tma = 0;
     }
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
-    static const int sk_threshold[6] = {/*GATEUP*/ 16, /*DOWN*/ 40, /*DH*/ 96, /*DW*/ 64, /*DX*/ 40, /*PLAIN*/ 32};
+    static const int sk_threshold[6] = {/*GATEUP*/ 16, /*DOWN*/ 40, /*DH*/ 48, /*DW*/ 64, /*DX*/ 40, /*PLAIN*/ 32};
     p.streamk = (g.sk_slots && g.sk_flags) ? (g.tune_streamk >= 0 ? g.tune_streamk : sk_threshold[epi]) : 0;
 
     const int tile_w = p.force_bn > 0 ? p.force_bn : BN;   // accumulator columns per tile
@@ -1570,6 +1654,7 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
         (void)cudaGetLastError();
         no_pairs[dev] = 1;
     }
+    p.gather = 0;   // the one-CTA shape stages up to 256 token rows per CTA: compacted copy only
     return dispatch<false>(dev, epi, tm, p, max_items(BM), s);
 }
 

@@ -132,11 +132,12 @@ def test_k_split_schedule_forced_on_and_off(min_saving, case):
     _compare(w, run(w, tune=dict(streamk=min_saving)), _oracle_all(w))
 
 
-@pytest.mark.parametrize("knob", ["one_box", "tma_stores"])
+@pytest.mark.parametrize("knob", ["one_box", "tma_stores", "gather"])
 @pytest.mark.parametrize("grad_fp32", [False, True])
 def test_alternative_load_and_store_paths_give_the_same_bits(knob, grad_fp32):
     # operand tiles fetched with one 3-D box or one 2-D box per piece; weight-gradient tiles written
-    # by TMA tile stores or per-lane stores.  Shapes: multiples of 64 (where the one-box loads
+    # by TMA tile stores or per-lane stores; token rows of gate/up and dH gathered from x / dout by
+    # tile::gather4 loads or read from the compacted copy.  Shapes: multiples of 64 (where the one-box loads
     # apply) and ragged ones (where the tile stores clip at the matrix edges).
     for w in (wl.small_case(27, "bf16", 512, 1024, 3, 20, 300, 0.5), wl.small_case(28, "bf16", 576, 1000, 3, 20, 200, 0.6)):
         ref = _oracle_all(w)
