@@ -20,6 +20,7 @@ template <typename T>
 __global__ void __launch_bounds__(SM_THREADS)
 k_row_rnorm(const T *__restrict__ X, float *__restrict__ rn, int64_t n, int C)
 {
+    pdl_enter();
     const int64_t i = (int64_t)blockIdx.x * (SM_THREADS / 32) + (threadIdx.x >> 5);
     if (i >= n) return;
     const int lane = threadIdx.x & 31;
@@ -37,6 +38,7 @@ k_row_rnorm(const T *__restrict__ X, float *__restrict__ rn, int64_t n, int C)
 // avg[i] = rn[i] * dot[i] / n, in place over dot
 __global__ void k_scale_avg(float *__restrict__ avg, const float *__restrict__ rn, int64_t n)
 {
+    pdl_enter();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) avg[i] = avg[i] * rn[i] / (float)n;
 }
@@ -46,6 +48,7 @@ __global__ void __launch_bounds__(256)
 k_rank_select(const float *__restrict__ avg, int64_t n, int k, uint8_t *__restrict__ drop,
               uint8_t *__restrict__ drop_inv)
 {
+    pdl_enter();
     __shared__ float tile[256];
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
     const float a = i < n ? avg[i] : 0.0f;
@@ -73,6 +76,7 @@ __global__ void __launch_bounds__(128)
 k_gather_unit_rows(const T *__restrict__ X, const float *__restrict__ rn, const int32_t *__restrict__ idx,
                    int64_t count, T *__restrict__ dst, int C)
 {
+    pdl_enter();
     const int64_t r = blockIdx.x;
     float v[4];
     if (r < count) {
@@ -95,6 +99,7 @@ __global__ void __launch_bounds__(SM_THREADS)
 k_assign(const float *__restrict__ sims, int64_t n_rest, int k, const int32_t *__restrict__ rest,
          const int32_t *__restrict__ kept, int32_t *__restrict__ assign)
 {
+    pdl_enter();
     const int64_t r = (int64_t)blockIdx.x * (SM_THREADS / 32) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (r < n_rest) {
@@ -122,6 +127,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 k_merge_rows(const T *__restrict__ X, const int32_t *__restrict__ assign, int64_t n, T *__restrict__ merged, int C)
 {
+    pdl_enter();
     __shared__ int32_t members[256];
     __shared__ int warp_cnt[8];
     const int j = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -213,22 +219,22 @@ static cudaError_t merge_t(const T *X, int64_t n, int C, int k, int dtype, int32
     const int64_t n_rest = n - k;
     cudaError_t e;
     // 1. average similarity
-    k_row_rnorm<T><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, m.rn, n, C);
+    launch_pdl(k_row_rnorm<T>, dim3((unsigned)((n + 7) / 8)), dim3(SM_THREADS), s, X, m.rn, n, C);
     dim3 g1((C + SP_COLS - 1) / SP_COLS, DG_CHUNKS);
-    k_weighted_rows<T, float><<<g1, SP_COLS * SP_LANES, 0, s>>>(X, m.rn, nullptr, 0, n, m.part, C);
-    k_sum_parts<float><<<(C + 255) / 256, 256, 0, s>>>(m.part, DG_CHUNKS, m.mean, C);
-    k_row_dots<T, float><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, m.mean, nullptr, 0, 0, m.avg, n, C);
-    k_scale_avg<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(m.avg, m.rn, n);
+    launch_pdl(k_weighted_rows<T, float>, dim3(g1), dim3(SP_COLS * SP_LANES), s, X, m.rn, nullptr, 0, n, m.part, C);
+    launch_pdl(k_sum_parts<float>, dim3((C + 255) / 256), dim3(256), s, m.part, DG_CHUNKS, m.mean, C);
+    launch_pdl(k_row_dots<T, float>, dim3((unsigned)((n + 7) / 8)), dim3(SM_THREADS), s, X, m.mean, nullptr, 0, 0, m.avg, n, C);
+    launch_pdl(k_scale_avg, dim3((unsigned)((n + 255) / 256)), dim3(256), s, m.avg, m.rn, n);
     // 2. the k most distinctive tokens, and the others, each as an ascending index list
-    k_rank_select<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(m.avg, n, k, m.drop, m.drop_inv);
+    launch_pdl(k_rank_select, dim3((unsigned)((n + 255) / 256)), dim3(256), s, m.avg, n, k, m.drop, m.drop_inv);
     if ((e = cudaMemsetAsync(m.status_k, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, s)) != cudaSuccess) return e;
     if ((e = launch_compact(m.drop, n, 0, m.kept, m.pos, m.status_k, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
     if ((e = launch_compact(m.drop_inv, n, 0, m.rest, m.pos, m.status_r, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
     if ((e = cudaMemcpyAsync(kept_out, m.kept, (size_t)k * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess) return e;
     // 3. assignment: unit rows, similarity GEMM, arg max
     if (n_rest > 0) {
-        k_gather_unit_rows<T><<<(unsigned)round_up(n_rest, ROW_PAD), 128, 0, s>>>(X, m.rn, m.rest, n_rest, (T *)m.Xa, C);
-        k_gather_unit_rows<T><<<(unsigned)round_up(k, ROW_PAD), 128, 0, s>>>(X, m.rn, m.kept, k, (T *)m.Xb, C);
+        launch_pdl(k_gather_unit_rows<T>, dim3((unsigned)round_up(n_rest, ROW_PAD)), dim3(128), s, X, m.rn, m.rest, n_rest, (T *)m.Xa, C);
+        launch_pdl(k_gather_unit_rows<T>, dim3((unsigned)round_up(k, ROW_PAD)), dim3(128), s, X, m.rn, m.kept, k, (T *)m.Xb, C);
         GemmArgs g;
         memset(&g, 0, sizeof(g));
         g.A = m.Xa; g.lda_m = C; g.lda_k = 1; g.a_outer = round_up(n_rest, ROW_PAD);
@@ -240,10 +246,10 @@ static cudaError_t merge_t(const T *X, int64_t n, int C, int k, int dtype, int32
         e = dtype == SKIPFFN_BF16 ? launch_umma_gemm(EPI_PLAIN, g, s) : launch_simt_gemm(EPI_DW, dtype, g, s);
         if (e != cudaSuccess) return e;
     }
-    k_assign<<<(unsigned)((max((int64_t)k, n_rest * 32) + SM_THREADS - 1) / SM_THREADS), SM_THREADS, 0, s>>>(
+    launch_pdl(k_assign, dim3((unsigned)((max((int64_t)k, n_rest * 32) + SM_THREADS - 1) / SM_THREADS)), dim3(SM_THREADS), s, 
         m.sims, n_rest, k, m.rest, m.kept, assign);
     // 4. merge
-    k_merge_rows<T><<<k, 256, 0, s>>>(X, assign, n, merged, C);
+    launch_pdl(k_merge_rows<T>, dim3(k), dim3(256), s, X, assign, n, merged, C);
     return cudaGetLastError();
 }
 

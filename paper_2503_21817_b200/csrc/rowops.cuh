@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(SM_THREADS)
 k_row_dots(const T *__restrict__ X, const TV *__restrict__ v, const int32_t *__restrict__ off, int n_seg,
            int per_segment, float *__restrict__ out, int64_t n, int C)
 {
+    pdl_enter();
     const int64_t i = (int64_t)blockIdx.x * (SM_THREADS / 32) + (threadIdx.x >> 5);
     if (i >= n) return;
     const int lane = threadIdx.x & 31;
@@ -53,6 +54,7 @@ __global__ void __launch_bounds__(SP_COLS * SP_LANES)
 k_weighted_rows(const T *__restrict__ X, const float *__restrict__ coef, const int32_t *__restrict__ off,
                 int seg_mode, int64_t n, TO *__restrict__ out, int C)
 {
+    pdl_enter();
     __shared__ float red[SP_LANES][SP_COLS];
     int64_t lo, hi;
     if (seg_mode) { lo = off[blockIdx.y]; hi = off[blockIdx.y + 1]; }
@@ -77,6 +79,7 @@ k_weighted_rows(const T *__restrict__ X, const float *__restrict__ coef, const i
 template <typename TO>
 __global__ void k_sum_parts(const float *__restrict__ part, int parts, TO *__restrict__ out, int C)
 {
+    pdl_enter();
     const int col = blockIdx.x * blockDim.x + threadIdx.x;
     if (col >= C) return;
     float s = 0.0f;

@@ -29,6 +29,7 @@ __device__ __forceinline__ float block_reduce(float v, float *red, bool is_max)
 __global__ void __launch_bounds__(SM_THREADS)
 k_segment_softmax(float *__restrict__ probs, const int32_t *__restrict__ off)
 {
+    pdl_enter();
     __shared__ float red[SM_THREADS / 32];
     const int lo = off[blockIdx.x], hi = off[blockIdx.x + 1];
     float mx = -INFINITY;
@@ -44,6 +45,7 @@ k_segment_softmax(float *__restrict__ probs, const int32_t *__restrict__ off)
 __global__ void __launch_bounds__(SM_THREADS)
 k_segment_dscore(float *__restrict__ a, const float *__restrict__ probs, const int32_t *__restrict__ off)
 {
+    pdl_enter();
     __shared__ float red[SM_THREADS / 32];
     const int lo = off[blockIdx.x], hi = off[blockIdx.x + 1];
     float t = 0.0f;
@@ -58,6 +60,7 @@ __global__ void __launch_bounds__(SM_THREADS)
 k_summary_dx(const T *__restrict__ dxs, const T *__restrict__ w, const float *__restrict__ probs,
              const float *__restrict__ ds, const int32_t *__restrict__ off, int n_seg, T *__restrict__ dX, int C)
 {
+    pdl_enter();
     const int64_t i = blockIdx.x;
     int lo = 0, hi = n_seg;
     while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (off[mid] <= i) lo = mid; else hi = mid; }
@@ -72,11 +75,11 @@ static cudaError_t fwd_t(const T *X, const int32_t *off, int n_seg, int64_t n, i
                          float *probs, cudaStream_t s)
 {
     if (n > 0) {
-        k_row_dots<T><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, w, off, n_seg, 0, probs, n, C);
-        k_segment_softmax<<<n_seg, SM_THREADS, 0, s>>>(probs, off);
+        launch_pdl(k_row_dots<T>, dim3((unsigned)((n + 7) / 8)), dim3(SM_THREADS), s, X, w, off, n_seg, 0, probs, n, C);
+        launch_pdl(k_segment_softmax, dim3(n_seg), dim3(SM_THREADS), s, probs, off);
     }
     dim3 grid((C + SP_COLS - 1) / SP_COLS, n_seg);     // empty segments write zeros
-    k_weighted_rows<T, T><<<grid, SP_COLS * SP_LANES, 0, s>>>(X, probs, off, 1, n, xs, C);
+    launch_pdl(k_weighted_rows<T, T>, dim3(grid), dim3(SP_COLS * SP_LANES), s, X, probs, off, 1, n, xs, C);
     return cudaGetLastError();
 }
 
@@ -87,15 +90,15 @@ static cudaError_t bwd_t(const T *X, const int32_t *off, int n_seg, int64_t n, i
 {
     float *ds = scratch, *part = scratch + ((n + 63) / 64) * 64;
     if (n > 0) {
-        k_row_dots<T><<<(unsigned)((n + 7) / 8), SM_THREADS, 0, s>>>(X, dxs, off, n_seg, 1, ds, n, C);
-        k_segment_dscore<<<n_seg, SM_THREADS, 0, s>>>(ds, probs, off);
-        if (dX) k_summary_dx<T><<<(unsigned)n, SM_THREADS, 0, s>>>(dxs, w, probs, ds, off, n_seg, dX, C);
+        launch_pdl(k_row_dots<T>, dim3((unsigned)((n + 7) / 8)), dim3(SM_THREADS), s, X, dxs, off, n_seg, 1, ds, n, C);
+        launch_pdl(k_segment_dscore, dim3(n_seg), dim3(SM_THREADS), s, ds, probs, off);
+        if (dX) launch_pdl(k_summary_dx<T>, dim3((unsigned)n), dim3(SM_THREADS), s, dxs, w, probs, ds, off, n_seg, dX, C);
     }
     if (dw) {
         dim3 grid((C + SP_COLS - 1) / SP_COLS, DG_CHUNKS);
-        k_weighted_rows<T, float><<<grid, SP_COLS * SP_LANES, 0, s>>>(X, ds, off, 0, n, part, C);
-        if (dw_fp32) k_sum_parts<float><<<(C + 255) / 256, 256, 0, s>>>(part, DG_CHUNKS, (float *)dw, C);
-        else k_sum_parts<T><<<(C + 255) / 256, 256, 0, s>>>(part, DG_CHUNKS, (T *)dw, C);
+        launch_pdl(k_weighted_rows<T, float>, dim3(grid), dim3(SP_COLS * SP_LANES), s, X, ds, off, 0, n, part, C);
+        if (dw_fp32) launch_pdl(k_sum_parts<float>, dim3((C + 255) / 256), dim3(256), s, part, DG_CHUNKS, (float *)dw, C);
+        else launch_pdl(k_sum_parts<T>, dim3((C + 255) / 256), dim3(256), s, part, DG_CHUNKS, (T *)dw, C);
     }
     return cudaGetLastError();
 }
