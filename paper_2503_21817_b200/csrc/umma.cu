@@ -710,9 +710,11 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
     // the same number of tiles but of equal width (320 tokens: 160 + 160 instead of 256 + 64), which
     // balances the workers and avoids a sliver whose operand loads would cost as much as a full tile's
     int tile_w = p.force_bn > 0 ? p.force_bn : BN;
-    if (TOK && p.force_bn <= 0 && n_tot > 0) {
-        const int n_tiles = (n_tot + BN - 1) / BN;
-        tile_w = ((n_tot / 16 + n_tiles - 1) / n_tiles) * 16;
+    if constexpr (TOK) {
+        if (p.force_bn <= 0 && n_tot > 0) {
+            const int n_tiles = (n_tot + BN - 1) / BN;
+            tile_w = ((n_tot / 16 + n_tiles - 1) / n_tiles) * 16;
+        }
     }
     // tiles of problem g: ids [g_first[g], g_first[g+1]); token problems run the column (token)
     // tile index fastest, so that tiles sharing a weight panel run at the same time
