@@ -217,6 +217,12 @@ skipffn_status skipffn_token_merge(const void *X, int64_t n, int32_t C, int32_t 
                                    int32_t *kept, int32_t *assign, void *merged, void *scratch,
                                    size_t scratch_bytes, void *stream);
 
+/* Synchronises `stream` and reads the status word the last skipffn_token_merge call on this scratch
+ * (same n, C, k, dtype) left behind: SKIPFFN_ETIMEOUT with the wait site in *site_out (may be NULL)
+ * if its tensor-core kernel gave up on a wait, else SKIPFFN_OK. */
+skipffn_status skipffn_token_merge_poll(void *scratch, int64_t n, int32_t C, int32_t k, int32_t dtype,
+                                        void *stream, int32_t *site_out);
+
 /* Device addresses of the kept-row index list (int32, ascending) and of its length. */
 skipffn_status skipffn_get_kept(const skipffn_saved *saved, const int32_t **idx_dev,
                                 const int32_t **nk_dev);

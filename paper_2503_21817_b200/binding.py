@@ -21,7 +21,8 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_forward_prenorm", "skipffn_backward_prenorm", "skipffn_summary_scratch_bytes",
            "skipffn_summary_forward", "skipffn_summary_backward", "skipffn_token_merge_scratch_bytes",
            "skipffn_token_merge", "skipffn_tune", "skipffn_saved_bytes", "skipffn_scratch_bytes",
-           "skipffn_workspace_bytes_kept", "skipffn_saved_create_kept", "skipffn_saved_create_split"]
+           "skipffn_workspace_bytes_kept", "skipffn_saved_create_kept", "skipffn_saved_create_split",
+           "skipffn_token_merge_poll"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4, "tma_stores": 5, "gather": 6}
@@ -109,6 +110,8 @@ def load_library() -> ctypes.CDLL:
     lib.skipffn_token_merge_scratch_bytes.argtypes = [i64, i32, i32, i32]
     lib.skipffn_token_merge.restype = i32
     lib.skipffn_token_merge.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.skipffn_token_merge_poll.restype = i32
+    lib.skipffn_token_merge_poll.argtypes = [vp, i64, i32, i32, i32, vp, ctypes.POINTER(i32)]
     lib.skipffn_strerror.restype = ctypes.c_char_p
     lib.skipffn_strerror.argtypes = [i32]
     _lib = lib
@@ -195,9 +198,11 @@ def summary_backward(X, seg_offsets, w, probs, dxs, dw_fp32=False):
     return dX, dw
 
 
-def token_merge(X, k: int):
+def token_merge(X, k: int, poll: bool = False):
     """Token merge of section 4.1 (``skipffn_token_merge``): ``(kept [k], assign [n], merged [k, C])``
-    for the tokens ``X [n, C]`` (bf16 or fp32 CUDA tensor)."""
+    for the tokens ``X [n, C]`` (bf16 or fp32 CUDA tensor).  ``poll=True`` synchronises the stream
+    afterwards and raises if the tensor-core kernel reported a timed-out wait
+    (``skipffn_token_merge_poll``)."""
     import torch
     lib = load_library()
     dtype = BF16 if X.dtype == torch.bfloat16 else FP32
@@ -212,6 +217,11 @@ def token_merge(X, k: int):
                                  ctypes.c_void_p(sp), nbytes, _stream_of(X))
     if st != 0:
         raise SkipFFNError(st, "skipffn_token_merge")
+    if poll:
+        site = ctypes.c_int32(0)
+        st = lib.skipffn_token_merge_poll(ctypes.c_void_p(sp), n, C, k, dtype, _stream_of(X), ctypes.byref(site))
+        if st != 0:
+            raise SkipFFNError(st, f"skipffn_token_merge_poll (site {site.value})")
     return kept, assign, merged
 
 

@@ -653,6 +653,19 @@ skipffn_status skipffn_token_merge(const void *X, int64_t n, int32_t C, int32_t 
                ? SKIPFFN_OK : SKIPFFN_ECUDA;
 }
 
+skipffn_status skipffn_token_merge_poll(void *scratch, int64_t n, int32_t C, int32_t k, int32_t dtype, void *stream,
+                                        int32_t *site_out)
+{
+    if (!scratch || n <= 0 || k <= 0 || k > n || C <= 0 || (dtype != SKIPFFN_BF16 && dtype != SKIPFFN_FP32))
+        return SKIPFFN_EINVAL;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return SKIPFFN_ECUDA;
+    int32_t w[3] = {0, 0, 0};
+    if (cudaMemcpy(w, merge_status_ptr(scratch, n, C, k, dtype), sizeof(w), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SKIPFFN_ECUDA;
+    if (site_out) *site_out = w[ST_SITE];
+    return (skipffn_status)w[ST_STATUS];
+}
+
 skipffn_status skipffn_get_kept(const skipffn_saved *s, const int32_t **idx_dev, const int32_t **nk_dev)
 {
     if (!s || s->planned_N < 0) return SKIPFFN_EINVAL;

@@ -185,6 +185,7 @@ cudaError_t launch_summary_backward(const void *X, const int32_t *off, int n_seg
                                     int dw_fp32, float *scratch, cudaStream_t s);
 // merge.cu
 size_t merge_scratch_bytes(int64_t n, int C, int k, int dtype);
+int32_t *merge_status_ptr(void *scratch, int64_t n, int C, int k, int dtype);
 cudaError_t launch_token_merge(const void *X, int64_t n, int C, int k, int dtype, int32_t *kept, int32_t *assign,
                                void *merged, void *scratch, cudaStream_t s);
 // simt.cu

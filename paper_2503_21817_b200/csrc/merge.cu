@@ -205,6 +205,12 @@ static MergeScratch merge_layout(char *base, int64_t n, int C, int k, int es)
     return m;
 }
 
+// device address of the status block the merge's tensor-core GEMM reports to (inside the scratch)
+int32_t *merge_status_ptr(void *scratch, int64_t n, int C, int k, int dtype)
+{
+    return merge_layout((char *)scratch, n, C, k, dtype == SKIPFFN_BF16 ? 2 : 4).status_k;
+}
+
 size_t merge_scratch_bytes(int64_t n, int C, int k, int dtype)
 {
     return merge_layout(nullptr, n, C, k, dtype == SKIPFFN_BF16 ? 2 : 4).total + (size_t)SK_MAX_CTAS * SK_SLOT_BYTES;

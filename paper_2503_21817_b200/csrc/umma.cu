@@ -826,7 +826,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             if (groups > 2) prefetch_tmap(&tmA3);
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            long long role_a = 0;
+            [[maybe_unused]] long long role_a = 0;
             for (int si = 0; ok && si < num_segs; ++si) {
                 const Seg sg = sched.get(si);
                 const TileLoc tl = locate(sg.tile);
@@ -908,8 +908,8 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             const uint64_t db0 = B_MN ? make_desc(tiles + A_BYTES, CHUNK_BYTES, 1024) : make_desc(tiles + A_BYTES, 16, 1024);
             const int k_tail = K - (kb_per_seg - 1) * BK;   // elements in the last K-block
             const int k_steps_last = k_tail < BK ? (k_tail + UMMA_K - 1) / UMMA_K : BK / UMMA_K;
-            long long role_full = 0, role_acc = 0;
-            const long long role_t0 = ROLE_CLOCK();
+            [[maybe_unused]] long long role_full = 0, role_acc = 0;
+            [[maybe_unused]] const long long role_t0 = ROLE_CLOCK();
             for (int si = 0; ok && si < num_segs; ++si) {
                 const Seg sg = sched.get(si);
                 const TileLoc tl = locate(sg.tile);
@@ -973,8 +973,8 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
         const int esz = p.out_fp32 ? 4 : 2;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        long long role_wait = 0;
-        const long long role_e0 = ROLE_CLOCK();
+        [[maybe_unused]] long long role_wait = 0;
+        [[maybe_unused]] const long long role_e0 = ROLE_CLOCK();
         // gate/up: warps of quarters 0, 1 hold gate rows, quarters 2, 3 the up rows of the same
         // indices; pair x = (quarter & 1) + 2 * half exchanges the up values through shared memory
         const int xpair = (quarter & 1) + 2 * half;
