@@ -732,18 +732,34 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
     const int num_n0 = (g_n[0] + tile_w - 1) / tile_w;
     auto pick = [](const int (&a)[3], int g) { return g == 2 ? a[2] : (g == 1 ? a[1] : a[0]); };
     struct TileLoc { int g, m0, n0, bn; };   // m0 in units of output rows (gate/up: intermediate indices)
+    // Order of the tiles of one problem: `nf` tiles along the fast axis, visited in bands of `band`
+    // of them; inside a band the fast index runs fastest, then the slow index.  A wave of W tiles
+    // then covers about band x W/band tiles, so the operand panels it touches (band + W/band of them,
+    // each K long) stay within L2 when K is large; with nf <= band it is the plain order.
+    auto raster = [](int t, int nf, int ns, int band, int &f, int &sl) {
+        const int per_band = band * ns;
+        const int b = t / per_band, f0 = b * band;
+        const int width = min(band, nf - f0);
+        const int r = t - b * per_band;
+        f = f0 + r % width;
+        sl = r / width;
+    };
     auto locate = [&](int tile) {
         TileLoc t;
-        if (TOK) {
+        int f, sl;
+        if (TOK) {   // token tiles fastest (tiles sharing a weight panel run together), in bands of 16
             t.g = 0;
-            t.m0 = (tile / num_n0) * M_UNIT;
-            t.n0 = (tile % num_n0) * tile_w;
+            raster(tile, num_n0, g_num_m[0], 16, f, sl);
+            t.m0 = sl * M_UNIT;
+            t.n0 = f * tile_w;
             t.bn = min(tile_w, n_tot - t.n0);
-        } else {
+        } else {     // weight gradients: row tiles fastest, in bands of 8
             t.g = tile >= g_first[2] ? 2 : (tile >= g_first[1] ? 1 : 0);
             const int local = tile - (t.g == 2 ? g_first[2] : (t.g == 1 ? g_first[1] : 0)), nm = pick(g_num_m, t.g);
-            t.m0 = (local % nm) * TILE_M;
-            t.n0 = (local / nm) * tile_w;
+            const int nn = (pick(g_n, t.g) + tile_w - 1) / tile_w;
+            raster(local, nm, nn, 8, f, sl);
+            t.m0 = f * TILE_M;
+            t.n0 = sl * tile_w;
             t.bn = tile_w;
         }
         return t;
