@@ -8,6 +8,12 @@
 // W_gate / W_up (dX) and for both operands of the weight-gradient GEMMs, whose reduction axis is the
 // compacted token axis.
 //
+// Token problems (gate/up, down, dH, dX) put the WEIGHT rows on the accumulator rows (A operand,
+// MMA M = 256 per SM pair) and the kept TOKENS on the accumulator columns (B operand, MMA N = any
+// multiple of 16 up to 256): the kept count is padded to 16 instead of 256.  Their outputs are
+// token-major, the transpose of the accumulator; the epilogue works in MMA-fragment layout and
+// transposes through shared memory (tcgen05.ld 16x256b, stmatrix / ldmatrix .trans).
+//
 // Two launch shapes share the code:
 //   PAIR   two CTAs of a cluster (an SM pair) compute one 256 x bn tile with cta_group::2 MMAs.
 //          Each CTA stages its own 128 rows of A and HALF of the B tile, so an SM pulls 32 KiB
@@ -16,13 +22,14 @@
 //          Used when the device cannot co-schedule pairs.
 //
 // Warp roles (320 threads per CTA, one CTA per SM):
-//   warp 0      TMA producer: fills the stage ring (128-byte swizzle)
+//   warp 0      TMA producer: fills the stage ring (128-byte swizzle), two or three box loads per stage
 //   warp 1      MMA issuer (the pair's leader CTA issues for both SMs): owns the tensor-memory
 //               allocation (512 columns = two 128 x 256 fp32 accumulators per SM), issues four K=16
 //               tcgen05.mma per stage, releases stages and publishes finished accumulators through
 //               tcgen05.commit
-//   warps 2..9  epilogue: read one accumulator (tcgen05.ld, one row per thread) while the MMA warp
-//               fills the other, apply the fused epilogue, write global memory
+//   warps 2..9  epilogue: read one accumulator (tcgen05.ld) while the MMA warp fills the other,
+//               apply the fused epilogue, write global memory (16-byte accesses, or TMA tile
+//               stores for the weight gradients)
 //
 // The kept-token count Nk lives in device memory, so tile counts are derived on the device and no
 // host synchronisation sits between mask compaction and the GEMMs.  Every wait (mbarrier or
