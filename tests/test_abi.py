@@ -58,6 +58,42 @@ def test_host_only_entry_points():
         lib.skipffn_saved_destroy(saved)
 
 
+def test_memory_modes_sizes_and_host_side_checks():
+    # host-only: saved / scratch sizes of the memory modes, handle creation over two buffers, knobs
+    import paper_2503_21817_b200 as sk
+    from paper_2503_21817_b200.binding import _cfg
+    lib = sk.load_library()
+    C, I, N, nk = 4096, 14336, 4928, 1472
+    plain, rec, dbg = _cfg(C, I), _cfg(C, I, recompute=True), _cfg(C, I, debug=True)
+    by = lambda fn, c, mk: int(fn(ctypes.byref(c), N, mk))
+    sv, sc, ws = lib.skipffn_saved_bytes, lib.skipffn_scratch_bytes, lib.skipffn_workspace_bytes_kept
+    # one buffer = saved + scratch; the classic size is the kept-sized one with max_kept = max_tokens
+    assert by(ws, plain, N) == by(sv, plain, N) + by(sc, plain, N) == sk.skipffn_workspace_bytes(C, I, N)
+    # compacted arrays scale with the kept bound: G, U, H (saved) and dG, dU, dOk (scratch)
+    assert by(sv, plain, nk) < 0.35 * by(sv, plain, N) and by(sc, plain, nk) < 0.4 * by(sc, plain, N)
+    assert by(sv, plain, nk) > 3 * 1536 * I * 2
+    # recompute: G, U, H move from saved to scratch; what is saved is the kept rows of x and two index arrays
+    assert by(sv, rec, nk) < 1536 * C * 2 + 2 * 5120 * 4 + 16384
+    assert by(sv, rec, nk) + by(sc, rec, nk) == by(sv, plain, nk) + by(sc, plain, nk)
+    # debug handles pay for their guard bands; invalid bounds give size 0
+    assert by(sv, dbg, nk) > by(sv, plain, nk)
+    assert by(sv, plain, N + 1) == 0 and int(sv(ctypes.byref(plain), -1, 0)) == 0
+    saved = ctypes.c_void_p()
+    a, b = ctypes.c_void_p(1 << 20), ctypes.c_void_p(1 << 30)
+    cr = lib.skipffn_saved_create_split
+    assert cr(ctypes.byref(saved), ctypes.byref(rec), a, by(sv, rec, nk) - 1, b, 1 << 40, N, nk) == 3    # saved too small
+    assert cr(ctypes.byref(saved), ctypes.byref(rec), a, 1 << 40, b, by(sc, rec, nk) - 1, N, nk) == 3    # scratch too small
+    assert cr(ctypes.byref(saved), ctypes.byref(rec), a, 1 << 40, None, 1 << 40, N, nk) == 1             # no scratch
+    assert cr(ctypes.byref(saved), ctypes.byref(rec), a, 1 << 40, b, 1 << 40, N, N + 1) == 1             # bound > tokens
+    assert cr(ctypes.byref(saved), ctypes.byref(rec), a, by(sv, rec, nk), b, by(sc, rec, nk), N, nk) == 0
+    try:
+        assert lib.skipffn_tune(saved, 0, 128) == 0 and lib.skipffn_tune(saved, 99, 1) == 1
+        assert lib.skipffn_tune(saved, sk.binding.TUNABLES["lose_handover"], 1) == 1                      # debug handles only
+    finally:
+        lib.skipffn_saved_destroy(saved)
+    assert lib.skipffn_token_merge_poll(None, 10, 64, 4, 0, None, None) == 1
+
+
 def test_no_cpu_fallback():
     import torch
     import paper_2503_21817_b200 as sk
