@@ -409,8 +409,8 @@ static skipffn_status forward_impl(skipffn_saved *s, const void *x, const uint8_
     const int32_t NB = (int32_t)(N < s->max_kept ? N : s->max_kept);   // host bound of the kept count
     const bool tc = use_umma(s);
     // a recomputing handle keeps only H (for the down projection); its backward computes G, U, H again
-    // (the gathering variant reads x itself, so it cannot be used when out aliases x: the down
-    // projection of an earlier tile may already have overwritten rows -- not here, gate/up ends first)
+    // (with the GATHER knob the launch reads its token rows from x itself; it ends before the down
+    // projection writes `out`, so out may still alias x)
     if (gate_up(s, SLOT_GATEUP, NB, !s->cfg.recompute, st, x, N) != cudaSuccess) return SKIPFFN_ECUDA;
 
     // out[idx[r]] = Xk[r] + H Wd^T

@@ -148,6 +148,17 @@ def test_alternative_load_and_store_paths_give_the_same_bits(knob, grad_fp32):
             assert np.array_equal(bits(a[k]), bits(b[k])), k
 
 
+@pytest.mark.parametrize("C,I", [(8, 8), (8, 24), (24, 40), (72, 136), (200, 328)])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_tiny_and_odd_layer_widths(C, I, dtype):
+    # widths far below one tile and one K-block, multiples of 8 only: every box reaches past the
+    # arrays' ends (zero fill on loads, clipping on tile stores)
+    w = wl.uniform_batch(61, dtype, C, I, 2, 3, 70, 2, skip_ratio=0.6)
+    _compare(w, run(w), _oracle_all(w))
+    if dtype == "bf16":
+        _compare(w, run(w, grad_fp32=True), _oracle_all(w))
+
+
 def test_contiguous_span_layout():
     # the paper's layout: one contiguous skipped span per sequence
     w = wl.uniform_batch(2, "bf16", 256, 512, 4, 10, 150, 10, skip_ratio=0.8, contiguous_span=True)
