@@ -121,13 +121,20 @@ void skipffn_saved_destroy(skipffn_saved *saved);
  *                   tile::gather4 TMA loads driven by the kept-row list, instead of from the
  *                   compacted copy (which is still made: the weight gradients and the residual
  *                   read it).  0 (default): compacted copy, which measured faster
+ *   PANEL_SYNC      down and dX GEMMs with few tiles and a long reduction: -1 (default) or 1: when it
+ *                   costs under 6 % more K-blocks per worker, the workers form groups of one per
+ *                   token tile and each group walks the K-blocks of a weight panel side by side,
+ *                   so that a panel is fetched from DRAM once (its loads carry an L2 evict-first
+ *                   policy, so that the token operand stays cached); 2: always; 0: every worker
+ *                   takes its own contiguous run of K-blocks; add 4 to 1 or 2 to leave the
+ *                   eviction policy off
  *   LOSE_HANDOVER   debug handles only (EINVAL otherwise): nonzero makes the finishing units of a
  *                   K-split launch wait for a hand-over that never comes, so that the bounded wait
  *                   runs out and skipffn_poll reports SKIPFFN_ETIMEOUT -- the failure path can be
  *                   exercised without any fault */
 typedef enum { SKIPFFN_TUNE_TILE_N = 0, SKIPFFN_TUNE_STREAMK = 1, SKIPFFN_TUNE_STAGES = 2,
                SKIPFFN_TUNE_LOSE_HANDOVER = 3, SKIPFFN_TUNE_ONE_BOX = 4, SKIPFFN_TUNE_TMA_STORES = 5, SKIPFFN_TUNE_GATHER = 6,
-               SKIPFFN_TUNE_COUNT = 7 } skipffn_tunable;
+               SKIPFFN_TUNE_PANEL_SYNC = 7, SKIPFFN_TUNE_COUNT = 8 } skipffn_tunable;
 skipffn_status skipffn_tune(skipffn_saved *saved, int32_t what, int32_t value);
 
 /* Mask compaction alone (the retained / skipped split is the same for every decoder layer, so a

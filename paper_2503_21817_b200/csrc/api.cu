@@ -154,6 +154,7 @@ GemmArgs base_args(skipffn_saved *s)
     g.tune_tile_n = s->tune[SKIPFFN_TUNE_TILE_N];
     g.tune_stages = s->tune[SKIPFFN_TUNE_STAGES];
     g.tune_streamk = s->tune[SKIPFFN_TUNE_STREAMK];
+    g.tune_panel_sync = s->tune[SKIPFFN_TUNE_PANEL_SYNC];
     // failure-path hook of debug handles: finishing units of a K-split launch wait for a hand-over
     // flag value that nothing writes, so their bounded wait runs out
     g.sk_wait_skew = (s->cfg.debug && s->tune[SKIPFFN_TUNE_LOSE_HANDOVER]) ? 0x40000000 : 0;
@@ -255,6 +256,7 @@ skipffn_status skipffn_saved_create_split(skipffn_saved **saved, const skipffn_c
     s->dg_part = (float *)(x + l.dg_part);
     s->planned_N = -1;
     s->tune[SKIPFFN_TUNE_STREAMK] = -1;
+    s->tune[SKIPFFN_TUNE_PANEL_SYNC] = -1;
     s->tune[SKIPFFN_TUNE_ONE_BOX] = 1;
     s->tune[SKIPFFN_TUNE_TMA_STORES] = 1;
     s->guards.n = l.n_guards;

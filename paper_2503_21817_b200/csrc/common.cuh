@@ -141,6 +141,7 @@ struct GemmArgs {
     int32_t sk_wait_skew;       // 0; debug handles: make finishing units wait for a value nobody writes
     // tensor-core path: tuning overrides of the handle (0 / -1 = defaults) and its tensor-map cache
     int32_t tune_tile_n, tune_stages, tune_streamk;
+    int32_t tune_panel_sync;    // down, dX: -1 choose, 0 never, 1 when cheap, 2 always group workers by weight panel
     int32_t one_box_loads;      // 1: load an operand tile with one 3-D box where the arrays allow it
     int32_t tma_stores;         // 1: weight-gradient tiles leave through TMA tile stores (overwrite mode)
     // gate/up, dH (tensor-core path): non-null = fetch the token operand from this [gather_rows, K]

@@ -45,7 +45,11 @@
 // workspace (each worker has at most one such run and processes it first); the worker whose run
 // contains the tile's final K-block adds the slots of its predecessors, in a fixed order, and
 // runs the epilogue.  The summation order depends only on the shapes, so results are
-// reproducible from run to run.
+// reproducible from run to run.  The down and dX launches at a high skip ratio (few tiles, hundreds
+// of K-blocks each) use the same schedule one level up: the workers form groups of one member per
+// token tile, a group takes the place of a worker and a weight panel (all token tiles of one row
+// block) the place of a tile, so the members of a group read the same weight bytes at the same time
+// and DRAM delivers them once.
 #include <cuda.h>
 #include <stdlib.h>
 #include <string.h>
@@ -450,6 +454,7 @@ struct UmmaParams {
     int64_t gldo[3];
     int32_t streamk;                 // 0: whole tiles only; else the least number of K-blocks per worker
                                      // that cutting the last waves along K must save to be used
+    int32_t panel_sync;              // down, dX: 1 = the token tiles of a weight panel run side by side (see kernel)
     // one-instruction operand loads (see TmapSet): which of them the host could encode
     int32_t a_one, b_one;            // MN-major operand: both 64-wide slabs of a CTA's 128 in one 3-D box
     int32_t gu_one;                  // gate/up: gate and up rows in one 3-D box; 2 = the up rows come first
@@ -781,8 +786,41 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
     const int rem_tiles = num_tiles % num_workers;
     const bool split_k = p.streamk > 0 && rem_tiles != 0 &&
                          (long long)(num_workers - rem_tiles) * num_kb >= (long long)p.streamk * num_workers;
-    sched.init(worker, num_workers, num_tiles, num_kb, split_k);
+    // Few tiles with a long K (down, dX at a high skip ratio): every worker would sit at a K offset of
+    // its own, and the token tiles that share a weight panel would read it at different times, each
+    // time from DRAM.  Instead the workers form groups of `gw` = one per token tile; a group walks the
+    // (panel, K-block) space as ONE worker of the schedule above, its members side by side on the
+    // same K-blocks of the same panel, so a panel byte is fetched from DRAM once and hit in L2 by the
+    // other gw-1 members.  Workers beyond the last whole group stay idle; the mode is used when that
+    // and the coarser balance cost less than 6 % more K-blocks per worker.
+    int gw = 1;
+    if (TOK && (EPI == EPI_DOWN || EPI == EPI_DX) && p.panel_sync && p.streamk > 0 && num_n0 >= 2 && num_n0 <= 16 &&
+        num_n0 <= num_workers && num_kb > 0) {
+        const int ng = num_workers / num_n0;
+        const long long plain = ((long long)num_tiles * num_kb + num_workers - 1) / num_workers;
+        const long long grouped = ((long long)g_num_m[0] * num_kb + ng - 1) / ng;
+        if (p.panel_sync == 2 || (num_tiles < 2 * num_workers && num_kb >= 32 && grouped * 100 <= plain * 106)) gw = num_n0;
+    }
+    const int gcol = gw > 1 ? worker % gw : 0;
+    if (gw > 1) {
+        const int ng = num_workers / gw, sw = worker / gw, np = g_num_m[0];
+        const int rem_p = np % ng;
+        const bool split_p = rem_p != 0 && (long long)(ng - rem_p) * num_kb >= (long long)p.streamk * ng;
+        if (sw < ng) sched.init(sw, ng, np, num_kb, split_p);
+        else sched.init(0, 1, 0, num_kb, false);   // spare worker: nothing to do
+    } else {
+        sched.init(worker, num_workers, num_tiles, num_kb, split_k);
+    }
     const int num_segs = sched.count();
+    // unit i of this worker; in group mode the schedule's tile is a weight panel and this worker takes
+    // its own token tile of it (token tiles are the fast index of the tile order)
+    auto seg_at = [&](int i) {
+        Seg sg = sched.get(i);
+        if (gw > 1) sg.tile = sg.tile * gw + gcol;
+        return sg;
+    };
+    // CTA slot of schedule worker q (same token tile, same CTA rank as this one)
+    auto slot_cta = [&](int q) { return (gw > 1 ? q * gw + gcol : q) * SPLIT + (int)rank; };
     const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
 
     if (warp == 0) {
@@ -794,7 +832,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int si = 0; ok && si < num_segs; ++si) {
-                const Seg sg = sched.get(si);
+                const Seg sg = seg_at(si);
                 const TileLoc tl = locate(sg.tile);
                 const int bn_cta = tl.bn / SPLIT;
                 const int rows4 = (bn_cta + 3) >> 2;                     // gather4 loads of this CTA per K-block
@@ -851,7 +889,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             bool ok = true;
             [[maybe_unused]] long long role_a = 0;
             for (int si = 0; ok && si < num_segs; ++si) {
-                const Seg sg = sched.get(si);
+                const Seg sg = seg_at(si);
                 const TileLoc tl = locate(sg.tile);
                 const int bn_cta = tl.bn / SPLIT;          // B rows (tile columns) this CTA stages
                 const int b_slabs = (bn_cta + 63) / 64;
@@ -934,7 +972,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             [[maybe_unused]] long long role_full = 0, role_acc = 0;
             [[maybe_unused]] const long long role_t0 = ROLE_CLOCK();
             for (int si = 0; ok && si < num_segs; ++si) {
-                const Seg sg = sched.get(si);
+                const Seg sg = seg_at(si);
                 const TileLoc tl = locate(sg.tile);
                 const uint32_t idesc = make_idesc(A_MN ? 1 : 0, B_MN ? 1 : 0, TILE_M, tl.bn);
                 const long long ta = ROLE_CLOCK();
@@ -1013,7 +1051,7 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             return p.sk_slots + (size_t)cta_slot * (SK_SLOT_BYTES / 16) + ((size_t)(ew * 4 + j) * 8) * 32 + lane;
         };
         for (int si = 0; ok && si < num_segs; ++si) {
-            const Seg sg = sched.get(si);
+            const Seg sg = seg_at(si);
             const TileLoc tl = locate(sg.tile);
             const int n0 = tl.n0, bn = tl.bn;
             if (sg.partial) {
@@ -1067,9 +1105,9 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
             if (add_slots) {
                 // the rest of this tile's K range sits in the slots of workers src_lo .. worker-1
-                for (int q = sg.src_lo; ok && q < worker; ++q) {
+                for (int q = sg.src_lo; ok && q < sched.w; ++q) {
                     if (sched.bound(q + 1) == sched.bound(q)) continue;   // that worker had no run
-                    ok = flag_wait(p.sk_flags + (q * SPLIT + (int)rank) * SK_FLAGS_PER_CTA + ew,
+                    ok = flag_wait(p.sk_flags + slot_cta(q) * SK_FLAGS_PER_CTA + ew,
                                    p.sk_epoch + p.sk_wait_skew, lane, abort_flag, p.status);
                 }
                 if (!ok) break;
@@ -1090,9 +1128,9 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
                 }
                 if (add_slots) {
                     const int j = col >> 6;   // this warp's j-th 32-column chunk of the accumulator
-                    for (int q = sg.src_lo; q < worker; ++q) {
+                    for (int q = sg.src_lo; q < sched.w; ++q) {
                         if (sched.bound(q + 1) == sched.bound(q)) continue;
-                        const float4 *src = slot_ptr(q * SPLIT + (int)rank, j);
+                        const float4 *src = slot_ptr(slot_cta(q), j);
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
                             const float4 a = __ldcg(src + v * 32);
@@ -1655,6 +1693,7 @@ static cudaError_t launch_problems(int epi, const GemmArgs *gs, int n, cudaStrea
     // K-blocks of main loop (about 512 cycles each) that two extra epilogues of this kind cost
     static const int sk_threshold[6] = {/*GATEUP*/ 16, /*DOWN*/ 40, /*DH*/ 48, /*DW*/ 64, /*DX*/ 40, /*PLAIN*/ 32};
     p.streamk = (g.sk_slots && g.sk_flags) ? (g.tune_streamk >= 0 ? g.tune_streamk : sk_threshold[epi]) : 0;
+    p.panel_sync = g.tune_panel_sync < 0 ? 1 : g.tune_panel_sync;
 
     const int tile_w = p.force_bn > 0 ? p.force_bn : BN;   // accumulator columns per tile
     // with K splitting a tile can be shared by several workers: allow one worker per 4 K-blocks

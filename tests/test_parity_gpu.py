@@ -132,6 +132,24 @@ def test_k_split_schedule_forced_on_and_off(min_saving, case):
     _compare(w, run(w, tune=dict(streamk=min_saving)), _oracle_all(w))
 
 
+@pytest.mark.parametrize("mode", [0, 2])
+@pytest.mark.parametrize("case", ["ragged", "long_k", "one_token_tile", "many_panels"])
+def test_down_and_dx_schedules_by_weight_panel_or_by_worker(case, mode):
+    # down and dX either give every worker its own run of K-blocks (0) or let groups of workers, one
+    # per token tile, walk a weight panel's K-blocks side by side (2 = always, also where the
+    # library would not choose it).  The partial sums are cut at different K-blocks, so the two agree
+    # with the oracle, not bit for bit with each other.
+    if case == "ragged":            # 3-4 token tiles, C not a multiple of the panel height
+        w = wl.small_case(31, "bf16", 576, 1000, 4, 30, 400, 0.55)
+    elif case == "long_k":          # 64 / 128 K-blocks, two panels, groups share them along K
+        w = wl.small_case(32, "bf16", 512, 4096, 2, 16, 300, 0.4)
+    elif case == "one_token_tile":  # fewer kept tokens than one tile: groups of one
+        w = wl.small_case(33, "bf16", 1024, 2048, 2, 16, 100, 0.7)
+    else:                           # more panels than groups: whole panels first, the rest cut along K
+        w = wl.small_case(34, "bf16", 8192, 256, 3, 16, 260, 0.3)
+    _compare(w, run(w, tune=dict(panel_sync=mode)), _oracle_all(w))
+
+
 @pytest.mark.parametrize("knob", ["one_box", "tma_stores", "gather"])
 @pytest.mark.parametrize("grad_fp32", [False, True])
 def test_alternative_load_and_store_paths_give_the_same_bits(knob, grad_fp32):
