@@ -666,10 +666,10 @@ def run_summary(args):
     err = float(np.linalg.norm(xs[:2].float().cpu().numpy() - ref_xs) / np.linalg.norm(ref_xs))
     gbs = moved / (ms * 1e-3) / 1e9
     print(json.dumps({"metric": "summary_token_fwd_bwd_rows_per_s", "value": n / (ms * 1e-3), "unit": "rows/s", "ms": ms,
-                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 8,
+                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 4,
                       "config": {"workload": f"{len(sizes)} segments (8 samples x [144 retained | 432 skipped]), "
                                              f"{n} rows, C={C}", "l2_policy": "X (38 MB) fits in L2: second reads hit L2"},
-                      "roofline": {"kernel": "summary forward+backward (8 launches)", "bound": "hbm", "achieved": gbs,
+                      "roofline": {"kernel": "summary forward+backward (4 launches)", "bound": "hbm", "achieved": gbs,
                                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
                                    "peak_source": pk["source"], "traffic": None},
                       "xs_rel_error_first_sample": err,

@@ -190,6 +190,7 @@ skipffn_status skipffn_backward_prenorm(const void *dout, skipffn_saved *saved, 
  * Backward for upstream gradient dxs [n_seg, C]: dX [n_rows, C] (may be NULL), dw [C] (may be NULL;
  * fp32 if dw_fp32 or dtype is fp32), both overwritten.  scratch: device memory of
  * skipffn_summary_scratch_bytes(n_rows, C) bytes, 16-byte aligned (EWORKSPACE if smaller).
+ * X, w, xs, dxs and dX start on 16-byte boundaries (EINVAL otherwise).
  * Scores, weights and all sums are fp32 in a fixed order; outputs are rounded once. */
 size_t skipffn_summary_scratch_bytes(int64_t n_rows, int32_t C);
 skipffn_status skipffn_summary_forward(const void *X, const int32_t *seg_offsets, int32_t n_seg,

@@ -610,7 +610,8 @@ static bool summary_args_ok(const void *X, const int32_t *off, int32_t n_seg, in
                             int32_t dtype, const void *w)
 {
     return n_seg >= 0 && n_rows >= 0 && n_rows < ((int64_t)1 << 31) && C > 0 && C % 8 == 0 &&
-           (dtype == SKIPFFN_BF16 || dtype == SKIPFFN_FP32) && w && (n_seg == 0 || off) && (n_rows == 0 || X);
+           (dtype == SKIPFFN_BF16 || dtype == SKIPFFN_FP32) && w && (n_seg == 0 || off) && (n_rows == 0 || X) &&
+           aligned16(X) && aligned16(w);
 }
 
 skipffn_status skipffn_summary_forward(const void *X, const int32_t *seg_offsets, int32_t n_seg, int64_t n_rows,
@@ -619,6 +620,7 @@ skipffn_status skipffn_summary_forward(const void *X, const int32_t *seg_offsets
 {
     if (!summary_args_ok(X, seg_offsets, n_seg, n_rows, C, dtype, w)) return SKIPFFN_EINVAL;
     if (n_seg > 0 && (!xs || (n_rows > 0 && !probs))) return SKIPFFN_EINVAL;
+    if (!aligned16(xs)) return SKIPFFN_EINVAL;
     return launch_summary_forward(X, seg_offsets, n_seg, n_rows, C, dtype, w, xs, probs, (cudaStream_t)stream) ==
                    cudaSuccess ? SKIPFFN_OK : SKIPFFN_ECUDA;
 }
@@ -630,6 +632,7 @@ skipffn_status skipffn_summary_backward(const void *X, const int32_t *seg_offset
 {
     if (!summary_args_ok(X, seg_offsets, n_seg, n_rows, C, dtype, w)) return SKIPFFN_EINVAL;
     if (n_seg > 0 && (!dxs || !scratch || (n_rows > 0 && !probs))) return SKIPFFN_EINVAL;
+    if (!aligned16(dxs) || !aligned16(dX)) return SKIPFFN_EINVAL;
     if (scratch_bytes < skipffn_summary_scratch_bytes(n_rows, C)) return SKIPFFN_EWORKSPACE;
     if (((uintptr_t)scratch & 15u) != 0) return SKIPFFN_EINVAL;
     return launch_summary_backward(X, seg_offsets, n_seg, n_rows, C, dtype, w, probs, dxs, dX, dw, dw_fp32,
