@@ -22,6 +22,8 @@ At N = 1 the same line carries, measured after and outside the headline timed re
   sweep      skip ratios {0, .25, .5, .75, .9, 1} at both shapes against the in-library dense
              comparator on the same inputs
   host_us_per_step  host time of the eight launches of one step (no synchronisation)
+  step_times median and best of 50 steps timed one by one, and a step with a cold L2
+  seeds      the same workload drawn from two more seeds
 (`--no-extras` leaves them out.)
 """
 from __future__ import annotations
@@ -399,6 +401,49 @@ def run_ours(args):
             step()
         extras["host_us_per_step"] = (time.perf_counter() - th) / 40 * 1e6
         torch.cuda.synchronize()
+        # 50 steps timed one by one (events around each step): median and best; then one step with a
+        # cold L2 (a 512 MB buffer is written first)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(50)]
+        for a, b in evs:
+            a.record()
+            step()
+            b.record()
+        torch.cuda.synchronize()
+        each = sorted(a.elapsed_time(b) for a, b in evs)
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        cold = []
+        for _ in range(3):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step()
+            b.record()
+            torch.cuda.synchronize()
+            cold.append(a.elapsed_time(b))
+        del flush
+        extras["step_times"] = {"steps": len(each), "median_ms": each[len(each) // 2], "best_ms": each[0],
+                                "cold_l2_ms": sorted(cold)[1],
+                                "note": "each step timed alone; cold_l2: median of 3 steps that follow a 512 MB write"}
+        # other seeds: new activations, gradients and mask positions (same kept count), same weights
+        seeds = {}
+        for sd in (1, 2):
+            ws = wl.config2(seed=args.seed + sd, skip_ratio=args.skip_ratio, C=C, I=I,
+                            weights=(w.W_gate, w.W_up, w.W_down)) if args.workload == "cfg2" else None
+            if ws is None:
+                break
+            xs_, ds_, ms_ = h_bf16(ws.x).to(dev), h_bf16(ws.dout).to(dev), torch.from_numpy(ws.skip_mask).to(dev)
+
+            def step_seed():
+                ctx.forward(xs_, ms_, Wg, Wu, Wd, out=out)
+                ctx.backward(ds_, dx=dx, dW_gate=dWg, dW_up=dWu, dW_down=dWd)
+            for _ in range(3):
+                step_seed()
+            t_sd, _, _ = timed(step_seed, args.steps)
+            seeds[str(args.seed + sd)] = {"ms_per_step": t_sd / args.steps, "kept_tokens": ws.n_kept}
+            del xs_, ds_, ms_
+        if seeds:
+            extras["seeds"] = seeds
+        ctx.poll()
         # sustained: the same step for at least 3 s, clocks sampled over that region
         n_sus = max(args.steps, int(np.ceil(args.sustained_seconds * 1e3 / ms_step)))
         sampler = ClockSampler(local)
