@@ -1070,8 +1070,10 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             const int n0 = tl.n0, bn = tl.bn;
             if (sg.partial) {
                 // ---- this run ends before the tile does: park the raw accumulator in this CTA's slot
+                const long long tw = ROLE_CLOCK();
                 ok = mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, p.status,
                                SITE_EPI_TMEM_FULL);
+                ROLE_ADD(role_wait, tw);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
