@@ -753,10 +753,10 @@ def run_merge(args):
     flops = 2.0 * (n - k) * k * C + 4.0 * n * C
     moved = (4.0 * n + k) * C * 2                      # X read by norms, mean, averages, gather and merge
     print(json.dumps({"metric": "token_merge_rows_per_s", "value": n / (ms * 1e-3), "unit": "rows/s", "ms": ms,
-                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 13,
+                      "dtype": "bf16", "data": "synthetic", "gpu_launches": 11,
                       "config": {"workload": f"{n} tokens of {clusters} noisy clusters, C={C}, keep {k}",
                                  "l2_policy": "X (19 MB) stays in L2 after the first pass"},
-                      "roofline": {"kernel": "token merge (13 launches)", "bound": "hbm",
+                      "roofline": {"kernel": "token merge (11 launches)", "bound": "hbm",
                                    "achieved": moved / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
                                    "frac": moved / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], "peak_source": pk["source"],
                                    "traffic": None, "gemm_tflops": flops / (ms * 1e-3) / 1e12},

@@ -35,27 +35,20 @@ k_row_rnorm(const T *__restrict__ X, float *__restrict__ rn, int64_t n, int C)
     if (lane == 0) rn[i] = ss > 0.0f ? rsqrtf(ss) : 0.0f;
 }
 
-// avg[i] = rn[i] * dot[i] / n, in place over dot
-__global__ void k_scale_avg(float *__restrict__ avg, const float *__restrict__ rn, int64_t n)
-{
-    pdl_enter();
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) avg[i] = avg[i] * rn[i] / (float)n;
-}
-
-// keep[i] = 0 (kept) if fewer than k tokens precede i under (avg, index), else 1; rest = 1 - keep
+// avg_i = rn[i] * dot[i] / n.  keep[i] = 0 (kept) if fewer than k tokens precede i under (avg, index),
+// else 1; rest = 1 - keep
 __global__ void __launch_bounds__(256)
-k_rank_select(const float *__restrict__ avg, int64_t n, int k, uint8_t *__restrict__ drop,
-              uint8_t *__restrict__ drop_inv)
+k_rank_select(const float *__restrict__ dot, const float *__restrict__ rn, int64_t n, int k,
+              uint8_t *__restrict__ drop, uint8_t *__restrict__ drop_inv)
 {
     pdl_enter();
     __shared__ float tile[256];
     const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-    const float a = i < n ? avg[i] : 0.0f;
+    const float a = i < n ? dot[i] * rn[i] / (float)n : 0.0f;
     int rank = 0;
     for (int64_t j0 = 0; j0 < n; j0 += 256) {
         __syncthreads();
-        if (j0 + threadIdx.x < n) tile[threadIdx.x] = avg[j0 + threadIdx.x];
+        if (j0 + threadIdx.x < n) tile[threadIdx.x] = dot[j0 + threadIdx.x] * rn[j0 + threadIdx.x] / (float)n;
         __syncthreads();
         const int lim = (int)(n - j0 < 256 ? n - j0 : 256);
         for (int t = 0; t < lim; ++t) {
@@ -70,14 +63,20 @@ k_rank_select(const float *__restrict__ avg, int64_t n, int k, uint8_t *__restri
     }
 }
 
-// dst[r] = x[idx[r]] * rn[idx[r]] for r < count, zeros up to the next multiple of ROW_PAD
+// Two row sets in one launch: CTAs below rows_a fill dst_a from idx_a, the others dst_b from idx_b.
+// dst[r] = x[idx[r]] * rn[idx[r]] for r < count, zeros up to the next multiple of ROW_PAD.
 template <typename T>
 __global__ void __launch_bounds__(128)
-k_gather_unit_rows(const T *__restrict__ X, const float *__restrict__ rn, const int32_t *__restrict__ idx,
-                   int64_t count, T *__restrict__ dst, int C)
+k_gather_unit_rows(const T *__restrict__ X, const float *__restrict__ rn, const int32_t *__restrict__ idx_a,
+                   int64_t count_a, int64_t rows_a, T *__restrict__ dst_a, const int32_t *__restrict__ idx_b,
+                   int64_t count_b, T *__restrict__ dst_b, int C)
 {
     pdl_enter();
-    const int64_t r = blockIdx.x;
+    const bool second = (int64_t)blockIdx.x >= rows_a;
+    const int64_t r = second ? (int64_t)blockIdx.x - rows_a : (int64_t)blockIdx.x;
+    const int32_t *idx = second ? idx_b : idx_a;
+    const int64_t count = second ? count_b : count_a;
+    T *dst = second ? dst_b : dst_a;
     float v[4];
     if (r < count) {
         const int64_t t = idx[r];
@@ -230,17 +229,17 @@ static cudaError_t merge_t(const T *X, int64_t n, int C, int k, int dtype, int32
     launch_pdl(k_weighted_rows<T, float>, dim3(g1), dim3(SP_COLS * SP_LANES), s, X, m.rn, nullptr, 0, n, m.part, C);
     launch_pdl(k_sum_parts<float>, dim3((C + 255) / 256), dim3(256), s, m.part, DG_CHUNKS, m.mean, C);
     launch_pdl(k_row_dots<T, float>, dim3((unsigned)((n + 7) / 8)), dim3(SM_THREADS), s, X, m.mean, nullptr, 0, 0, m.avg, n, C);
-    launch_pdl(k_scale_avg, dim3((unsigned)((n + 255) / 256)), dim3(256), s, m.avg, m.rn, n);
     // 2. the k most distinctive tokens, and the others, each as an ascending index list
-    launch_pdl(k_rank_select, dim3((unsigned)((n + 255) / 256)), dim3(256), s, m.avg, n, k, m.drop, m.drop_inv);
+    launch_pdl(k_rank_select, dim3((unsigned)((n + 255) / 256)), dim3(256), s, m.avg, m.rn, n, k, m.drop, m.drop_inv);
     if ((e = cudaMemsetAsync(m.status_k, 0, (ST_WORDS + SK_FLAG_WORDS) * 4, s)) != cudaSuccess) return e;
     if ((e = launch_compact(m.drop, n, 0, m.kept, m.pos, m.status_k, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
     if ((e = launch_compact(m.drop_inv, n, 0, m.rest, m.pos, m.status_r, round_up(n, ROW_PAD) + ROW_PAD, n, s)) != cudaSuccess) return e;
     if ((e = cudaMemcpyAsync(kept_out, m.kept, (size_t)k * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess) return e;
     // 3. assignment: unit rows, similarity GEMM, arg max
     if (n_rest > 0) {
-        launch_pdl(k_gather_unit_rows<T>, dim3((unsigned)round_up(n_rest, ROW_PAD)), dim3(128), s, X, m.rn, m.rest, n_rest, (T *)m.Xa, C);
-        launch_pdl(k_gather_unit_rows<T>, dim3((unsigned)round_up(k, ROW_PAD)), dim3(128), s, X, m.rn, m.kept, k, (T *)m.Xb, C);
+        const int64_t rows_a = round_up(n_rest, ROW_PAD), rows_b = round_up(k, ROW_PAD);
+        launch_pdl(k_gather_unit_rows<T>, dim3((unsigned)(rows_a + rows_b)), dim3(128), s, X, m.rn, m.rest, n_rest, rows_a,
+                   (T *)m.Xa, m.kept, (int64_t)k, (T *)m.Xb, C);
         GemmArgs g;
         memset(&g, 0, sizeof(g));
         g.A = m.Xa; g.lda_m = C; g.lda_k = 1; g.a_outer = round_up(n_rest, ROW_PAD);
