@@ -298,6 +298,17 @@ int32_t skipffn_last_launches(const skipffn_saved *saved, int32_t which);
 int32_t skipffn_schedule_segment(int32_t workers, int32_t tiles, int32_t k_blocks, int32_t split_k,
                                  int32_t worker, int32_t i, int32_t *seg);
 
+/* Diagnostic (host only, launches nothing): the same for a token problem of `panels` blocks of weight
+ * rows x `token_tiles` token tiles (tile = panel * token_tiles + token tile), including the worker
+ * groups of the down / dX launches (group_mode as the PANEL_SYNC knob, min_saving as the STREAMK
+ * knob: least K-blocks per worker a cut must save, 0 = never cut).  seg[6] = {tile, first K-block,
+ * end K-block, partial, first source worker, source stride}: a finishing segment that starts at a
+ * K-block > 0 adds the accumulators handed over by workers seg[4], seg[4] + seg[5], ... below
+ * `worker` (those that have a partial segment of this tile). */
+int32_t skipffn_schedule_plan_segment(int32_t workers, int32_t panels, int32_t token_tiles, int32_t k_blocks,
+                                      int32_t min_saving, int32_t group_mode, int32_t worker, int32_t i,
+                                      int32_t *seg);
+
 /* Algorithmic floating-point operations of one forward+backward call with n_kept kept tokens:
  * 18 * n_kept * C * I (forward 6: three GEMMs of the section 6.2 cost model; backward 12). */
 double skipffn_flops(const skipffn_config *cfg, int64_t n_kept);

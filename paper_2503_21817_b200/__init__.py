@@ -6,7 +6,7 @@ with their fused epilogues) runs in the library's own kernels.  There is no CPU 
 fallback: if the library is missing, or no CUDA device is present, calls raise.
 """
 from .binding import (SkipFFNError, SkipFFN, load_library, skipffn_workspace_bytes, skipffn_flops,
-                      skipffn_strerror, skipffn_compact_static, skipffn_schedule, summary_forward, summary_backward, token_merge, STATIC_MAX_TOKENS, BF16, FP32, PATH_DEFAULT, PATH_SIMT, EXPORTS)
+                      skipffn_strerror, skipffn_compact_static, skipffn_schedule, skipffn_schedule_plan, summary_forward, summary_backward, token_merge, STATIC_MAX_TOKENS, BF16, FP32, PATH_DEFAULT, PATH_SIMT, EXPORTS)
 
 __all__ = ["SkipFFNError", "SkipFFN", "load_library", "skipffn_workspace_bytes", "skipffn_flops",
-           "skipffn_strerror", "skipffn_compact_static", "skipffn_schedule", "summary_forward", "summary_backward", "token_merge", "STATIC_MAX_TOKENS", "BF16", "FP32", "PATH_DEFAULT", "PATH_SIMT", "EXPORTS"]
+           "skipffn_strerror", "skipffn_compact_static", "skipffn_schedule", "skipffn_schedule_plan", "summary_forward", "summary_backward", "token_merge", "STATIC_MAX_TOKENS", "BF16", "FP32", "PATH_DEFAULT", "PATH_SIMT", "EXPORTS"]

@@ -22,7 +22,7 @@ EXPORTS = ["skipffn_workspace_bytes", "skipffn_saved_create", "skipffn_saved_des
            "skipffn_summary_forward", "skipffn_summary_backward", "skipffn_token_merge_scratch_bytes",
            "skipffn_token_merge", "skipffn_tune", "skipffn_saved_bytes", "skipffn_scratch_bytes",
            "skipffn_workspace_bytes_kept", "skipffn_saved_create_kept", "skipffn_saved_create_split",
-           "skipffn_token_merge_poll"]
+           "skipffn_token_merge_poll", "skipffn_schedule_plan_segment"]
 STATIC_MAX_TOKENS = 65536   # SKIPFFN_STATIC_MAX_TOKENS
 
 TUNABLES = {"tile_n": 0, "streamk": 1, "stages": 2, "lose_handover": 3, "one_box": 4, "tma_stores": 5, "gather": 6,
@@ -150,6 +150,23 @@ def skipffn_schedule(workers: int, tiles: int, k_blocks: int, split_k: bool, wor
     out = []
     for i in range(n):
         lib.skipffn_schedule_segment(workers, tiles, k_blocks, int(split_k), worker, i, seg)
+        out.append(tuple(seg))
+    return out
+
+
+def skipffn_schedule_plan(workers: int, panels: int, token_tiles: int, k_blocks: int, min_saving: int,
+                          group_mode: int, worker: int):
+    """Segments ``(tile, kb0, kb1, partial, first_source_worker, source_stride)`` of one worker's
+    schedule of a token problem, worker groups included (``skipffn_schedule_plan_segment``; host only)."""
+    lib = load_library()
+    seg = (ctypes.c_int32 * 6)()
+    args = (workers, panels, token_tiles, k_blocks, min_saving, group_mode, worker)
+    n = lib.skipffn_schedule_plan_segment(*args, -1, seg)
+    if n < 0:
+        raise SkipFFNError(1, "skipffn_schedule_plan_segment")
+    out = []
+    for i in range(n):
+        lib.skipffn_schedule_plan_segment(*args, i, seg)
         out.append(tuple(seg))
     return out
 

@@ -2,6 +2,8 @@
 #include <new>
 #include <string.h>
 
+#include <limits.h>
+
 #include "common.cuh"
 #include "sched.cuh"
 
@@ -719,6 +721,24 @@ int32_t skipffn_schedule_segment(int32_t workers, int32_t tiles, int32_t k_block
     if (seg && i >= 0 && i < n) {
         const Seg g = sc.get(i);
         seg[0] = g.tile; seg[1] = g.kb0; seg[2] = g.kb1; seg[3] = g.partial; seg[4] = g.src_lo;
+    }
+    return n;
+}
+
+int32_t skipffn_schedule_plan_segment(int32_t workers, int32_t panels, int32_t token_tiles, int32_t k_blocks,
+                                      int32_t min_saving, int32_t group_mode, int32_t worker, int32_t i, int32_t *seg)
+{
+    if (workers <= 0 || panels < 0 || token_tiles <= 0 || k_blocks < 0 || worker < 0 || worker >= workers ||
+        (int64_t)panels * token_tiles > INT_MAX)
+        return -1;
+    Plan pl;
+    pl.init(worker, workers, panels, token_tiles, k_blocks, min_saving, group_mode);
+    const int n = pl.count();
+    if (seg && i >= 0 && i < n) {
+        const Seg g = pl.get(i);
+        seg[0] = g.tile; seg[1] = g.kb0; seg[2] = g.kb1; seg[3] = g.partial;
+        seg[4] = pl.slot_worker(g.src_lo);
+        seg[5] = pl.gw;
     }
     return n;
 }

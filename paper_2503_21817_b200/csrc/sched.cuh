@@ -73,4 +73,57 @@ struct Sched {
     }
 };
 
+// Whether cutting the last waves along K pays: the idle time it removes, (W - T mod W) / W of a
+// tile's main loop, must be worth `min_saving` K-blocks per worker (0 = never cut).
+SKIPFFN_HD bool split_pays(int T, int W, int KB, int min_saving)
+{
+    const int rem = T % W;
+    return min_saving > 0 && rem != 0 && (long long)(W - rem) * KB >= (long long)min_saving * W;
+}
+
+// The schedule of one worker of a launch, with the worker groups of the down / dX launches.
+// Token problems order their tiles with the token-tile index fastest: tile = panel * n_tok + column,
+// a panel being all token tiles of one block of weight rows.  With groups (gw = n_tok > 1) the
+// W workers form W / gw groups of gw; a group takes the place of a worker and a panel the place of
+// a tile in `Sched`, and member `col` of a group works on token tile `col` of whatever panel and
+// K range its group has, so the members read the same weight bytes at the same time.  Workers
+// beyond the last whole group get nothing.  Hand-overs go from member `col` of one group to member
+// `col` of the next: schedule worker q of `src_lo .. w-1` is real worker slot_worker(q).
+struct Plan {
+    Sched s;
+    int gw, col;
+    // group_mode: 0 never, 1 when all tiles would be cut anyway (T < 2W), K has at least 32 blocks
+    // and groups cost under 6 % more K-blocks per worker, 2 always (n_tok between 2 and 16, <= W)
+    SKIPFFN_HD void init(int worker, int W, int panels, int n_tok, int KB, int min_saving, int group_mode)
+    {
+        const int T = panels * n_tok;
+        gw = 1;
+        if (group_mode && min_saving > 0 && n_tok >= 2 && n_tok <= 16 && n_tok <= W && KB > 0) {
+            const int ng = W / n_tok;
+            const long long plain = ((long long)T * KB + W - 1) / W;
+            const long long grouped = ((long long)panels * KB + ng - 1) / ng;
+            if (group_mode == 2 || (T < 2 * W && KB >= 32 && grouped * 100 <= plain * 106)) gw = n_tok;
+        }
+        col = gw > 1 ? worker % gw : 0;
+        if (gw > 1) {
+            const int ng = W / gw, sw = worker / gw;
+            if (sw < ng) s.init(sw, ng, panels, KB, split_pays(panels, ng, KB, min_saving));
+            else s.init(0, 1, 0, KB, 0);   // spare worker: nothing to do
+        } else {
+            s.init(worker, W, T, KB, split_pays(T, W, KB, min_saving));
+        }
+    }
+    SKIPFFN_HD int count() const { return s.count(); }
+    SKIPFFN_HD Seg get(int i) const
+    {
+        Seg sg = s.get(i);
+        if (gw > 1) sg.tile = sg.tile * gw + col;
+        return sg;
+    }
+    // real worker behind schedule worker q (a hand-over source of this worker)
+    SKIPFFN_HD int slot_worker(int q) const { return gw > 1 ? q * gw + col : q; }
+    SKIPFFN_HD bool had_run(int q) const { return s.bound(q + 1) != s.bound(q); }
+    SKIPFFN_HD int self() const { return s.w; }
+};
+
 }  // namespace skipffn

@@ -793,48 +793,21 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
     const int kb_per_seg = (K + BK - 1) / BK;
     const int num_kb = kb_per_seg * p.segments;
     const bool zero_acc = (num_kb == 0);   // empty reduction: the accumulator is exactly zero
-    Sched sched;
-    // Cutting the last waves costs every worker about two extra epilogues (one hand-over, one
-    // finish with the slot added); it pays when the idle time it removes, (W - T mod W) / W of a
-    // tile's main loop, is longer than that.
-    const int rem_tiles = num_tiles % num_workers;
-    const bool split_k = p.streamk > 0 && rem_tiles != 0 &&
-                         (long long)(num_workers - rem_tiles) * num_kb >= (long long)p.streamk * num_workers;
-    // Few tiles with a long K (down, dX at a high skip ratio): every worker would sit at a K offset of
-    // its own, and the token tiles that share a weight panel would read it at different times, each
-    // time from DRAM.  Instead the workers form groups of `gw` = one per token tile; a group walks the
-    // (panel, K-block) space as ONE worker of the schedule above, its members side by side on the
-    // same K-blocks of the same panel, so a panel byte is fetched from DRAM once and hit in L2 by the
-    // other gw-1 members.  Workers beyond the last whole group stay idle; the mode is used when that
-    // and the coarser balance cost less than 6 % more K-blocks per worker.
-    int gw = 1;
-    if (TOK && (EPI == EPI_DOWN || EPI == EPI_DX) && p.panel_sync && p.streamk > 0 && num_n0 >= 2 && num_n0 <= 16 &&
-        num_n0 <= num_workers && num_kb > 0) {
-        const int ng = num_workers / num_n0;
-        const long long plain = ((long long)num_tiles * num_kb + num_workers - 1) / num_workers;
-        const long long grouped = ((long long)g_num_m[0] * num_kb + ng - 1) / ng;
-        if (p.panel_sync == 2 || (num_tiles < 2 * num_workers && num_kb >= 32 && grouped * 100 <= plain * 106)) gw = num_n0;
-    }
-    const int gcol = gw > 1 ? worker % gw : 0;
-    if (gw > 1) {
-        const int ng = num_workers / gw, sw = worker / gw, np = g_num_m[0];
-        const int rem_p = np % ng;
-        const bool split_p = rem_p != 0 && (long long)(ng - rem_p) * num_kb >= (long long)p.streamk * ng;
-        if (sw < ng) sched.init(sw, ng, np, num_kb, split_p);
-        else sched.init(0, 1, 0, num_kb, false);   // spare worker: nothing to do
-    } else {
-        sched.init(worker, num_workers, num_tiles, num_kb, split_k);
-    }
+    // Work distribution (sched.cuh).  Cutting the last waves along K costs every worker about two
+    // extra epilogues (one hand-over, one finish with the slot added); it pays when the idle time it
+    // removes is longer than that (p.streamk K-blocks per worker).  Few tiles with a long K (down,
+    // dX at a high skip ratio): with one run per worker the token tiles that share a weight panel
+    // would sit at different K offsets and read the panel at different times, each time from DRAM;
+    // there the workers form groups that walk a panel's K-blocks side by side, so that a panel byte
+    // is fetched from DRAM once and hit in L2 by the other members.
+    Plan sched;
+    if (TOK) sched.init(worker, num_workers, g_num_m[0], num_n0, num_kb, p.streamk,
+                        (EPI == EPI_DOWN || EPI == EPI_DX) ? p.panel_sync : 0);
+    else sched.init(worker, num_workers, num_tiles, 1, num_kb, p.streamk, 0);
     const int num_segs = sched.count();
-    // unit i of this worker; in group mode the schedule's tile is a weight panel and this worker takes
-    // its own token tile of it (token tiles are the fast index of the tile order)
-    auto seg_at = [&](int i) {
-        Seg sg = sched.get(i);
-        if (gw > 1) sg.tile = sg.tile * gw + gcol;
-        return sg;
-    };
+    auto seg_at = [&](int i) { return sched.get(i); };
     // CTA slot of schedule worker q (same token tile, same CTA rank as this one)
-    auto slot_cta = [&](int q) { return (gw > 1 ? q * gw + gcol : q) * SPLIT + (int)rank; };
+    auto slot_cta = [&](int q) { return sched.slot_worker(q) * SPLIT + (int)rank; };
     const uint32_t nst = (p.force_stages > 0 && p.force_stages < STAGES) ? p.force_stages : STAGES;
 
     if (warp == 0) {
@@ -1148,8 +1121,8 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * ACC_COLS;
             if (add_slots) {
                 // the rest of this tile's K range sits in the slots of workers src_lo .. worker-1
-                for (int q = sg.src_lo; ok && q < sched.w; ++q) {
-                    if (sched.bound(q + 1) == sched.bound(q)) continue;   // that worker had no run
+                for (int q = sg.src_lo; ok && q < sched.self(); ++q) {
+                    if (!sched.had_run(q)) continue;
                     ok = flag_wait(p.sk_flags + slot_cta(q) * SK_FLAGS_PER_CTA + ew,
                                    p.sk_epoch + p.sk_wait_skew, lane, abort_flag, p.status);
                 }
@@ -1170,8 +1143,8 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
                 }
                 if (add_slots) {
                     const int j = col >> 6;   // this warp's j-th 32-column chunk of the accumulator
-                    for (int q = sg.src_lo; q < sched.w; ++q) {
-                        if (sched.bound(q + 1) == sched.bound(q)) continue;
+                    for (int q = sg.src_lo; q < sched.self(); ++q) {
+                        if (!sched.had_run(q)) continue;
                         const float4 *src = slot_ptr(slot_cta(q), j);
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
