@@ -23,6 +23,7 @@ At N = 1 the same line carries, measured after and outside the headline timed re
              comparator on the same inputs
   host_us_per_step  host time of the eight launches of one step (no synchronisation)
   step_times median and best of 50 steps timed one by one, and a step with a cold L2
+  graph_replay  the same step replayed from a captured CUDA graph
   seeds      the same workload drawn from two more seeds
 (`--no-extras` leaves them out.)
 """
@@ -424,6 +425,30 @@ def run_ours(args):
         extras["step_times"] = {"steps": len(each), "median_ms": each[len(each) // 2], "best_ms": each[0],
                                 "cold_l2_ms": sorted(cold)[1],
                                 "note": "each step timed alone; cold_l2: median of 3 steps that follow a 512 MB write"}
+        # the same step replayed from a CUDA graph (one host call per step instead of eight launches)
+        try:
+            cap = torch.cuda.Stream(dev)
+            cap.wait_stream(torch.cuda.current_stream(dev))
+            with torch.cuda.stream(cap):
+                step()
+            torch.cuda.current_stream(dev).wait_stream(cap)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            for _ in range(3):
+                graph.replay()
+            ms_g, _, _ = timed(graph.replay, args.steps)
+            torch.cuda.synchronize()
+            th = time.perf_counter()
+            for _ in range(40):
+                graph.replay()
+            host_g = (time.perf_counter() - th) / 40 * 1e6
+            torch.cuda.synchronize()
+            extras["graph_replay"] = {"ms_per_step": ms_g / args.steps, "host_us_per_step": host_g}
+            del graph
+        except Exception as exc:      # capture is a convenience of the harness, not part of the metric
+            extras["graph_replay"] = {"error": str(exc)[:200]}
         # other seeds: new activations, gradients and mask positions (same kept count), same weights
         seeds = {}
         for sd in (1, 2):

@@ -22,6 +22,13 @@
  *   - All work is enqueued on `stream`; the kept-token count stays on the device.
  *   - Device-side problems (a pipeline wait that exceeded its limit) set a status word in the
  *     workspace; the kernel then exits normally and skipffn_poll reports it.
+ *   - Stream capture: skipffn_plan, skipffn_forward and skipffn_backward only enqueue kernels and
+ *     asynchronous memsets on `stream`, so a forward + backward may be captured into a CUDA graph
+ *     after one un-captured call of the same sequence on the same handle (which does the one-time
+ *     work: kernel attributes, tensor-map encoding, clearing the status block).  A replay repeats
+ *     the captured kernel arguments, including the buffers the capture was given, and gives the
+ *     bits of the un-captured call; skipffn_poll and skipffn_profile_read synchronise and stay
+ *     outside a capture.
  */
 #ifndef SKIPFFN_H_
 #define SKIPFFN_H_

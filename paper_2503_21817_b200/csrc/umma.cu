@@ -1365,6 +1365,13 @@ k_umma_gemm(const __grid_constant__ TmapSet tm, const UmmaParams p)
                 }
             }
             if (!ok) break;
+            if (add_slots && lane == 0) {
+                // this warp has consumed the hand-overs of the tile: clear their flags, so that a replay
+                // of the launch with the same flag value (a captured graph) never takes an old flag for
+                // a new one
+                for (int q = sg.src_lo; q < sched.self(); ++q)
+                    if (sched.had_run(q)) p.sk_flags[slot_cta(q) * SK_FLAGS_PER_CTA + ew] = 0;
+            }
             if (!zero_acc) {
                 tc_fence_before();
                 __syncwarp();

@@ -319,6 +319,45 @@ def test_run_twice_bit_identical(tune):
         assert np.array_equal(bits(a[k]), bits(b[k])), k
 
 
+@pytest.mark.parametrize("tune", [None, dict(streamk=1, panel_sync=2)])
+def test_step_captured_in_a_cuda_graph_replays_the_same_bits(tune):
+    # the library never synchronises, allocates or reads back inside a call, so one forward +
+    # backward can be captured into a CUDA graph; every replay repeats the launches with the kernel
+    # arguments of the capture (the same hand-over flag values too) and must give the eager bits
+    import torch
+    sk = _sk()
+    w = wl.small_case(19, "bf16", 576, 2048, 3, 20, 200, 0.6)
+    d = DeviceWorkload(w)
+    ctx = sk.SkipFFN(w.C, w.I, w.N)
+    if tune:
+        ctx.tune(**tune)
+    out, dx = torch.empty_like(d.x), torch.empty_like(d.x)
+    dW = [torch.empty_like(t) for t in (d.W_gate, d.W_up, d.W_down)]
+
+    def step():
+        ctx.forward(d.x, d.mask, d.W_gate, d.W_up, d.W_down, out=out)
+        ctx.backward(d.dout, dx=dx, dW_gate=dW[0], dW_up=dW[1], dW_down=dW[2])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):       # warm-up on the side stream: first-use work happens outside the capture
+        step()
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    eager = [bits(t).copy() for t in (out, dx, *dW)]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for _ in range(3):
+        for t in (out, dx, *dW):
+            t.fill_(7.0)
+        g.replay()
+        torch.cuda.synchronize()
+        for a, t in zip(eager, (out, dx, *dW)):
+            assert np.array_equal(a, bits(t))
+    ctx.poll()
+
+
 def test_unsupported_and_invalid_arguments():
     import torch
     sk = _sk()
